@@ -1,0 +1,826 @@
+// C ABI of the Encode-stage library: handle, weight re-layout, workspace plan, and the launch
+// sequence of one micro-batch forward pass.  All arithmetic runs in the kernels included below.
+#include "../../include/eas_encoder.h"
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <cudaTypedefs.h>
+
+#include <algorithm>
+#include <cmath>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <map>
+#include <memory>
+#include <string>
+#include <vector>
+
+#include "attention_mma.cuh"
+#include "elementwise.cuh"
+#include "gemm.cuh"
+
+using namespace eas;
+
+// ------------------------------------------------------------------------------------ errors
+static thread_local char g_err[512] = "";
+static eas_status fail(eas_status s, const char* fmt, ...) {
+  va_list ap;
+  va_start(ap, fmt);
+  vsnprintf(g_err, sizeof(g_err), fmt, ap);
+  va_end(ap);
+  return s;
+}
+#define CUDA_TRY(expr)                                                                              \
+  do {                                                                                              \
+    cudaError_t e_ = (expr);                                                                        \
+    if (e_ != cudaSuccess) return fail(EAS_ERR_CUDA, "%s failed: %s", #expr, cudaGetErrorString(e_)); \
+  } while (0)
+
+extern "C" const char* eas_last_error(void) { return g_err; }
+
+// ------------------------------------------------------------------------------------ tensor maps
+static PFN_cuTensorMapEncodeTiled_v12000 get_encode_fn() {
+  static PFN_cuTensorMapEncodeTiled_v12000 fn = nullptr;
+  if (fn == nullptr) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<PFN_cuTensorMapEncodeTiled_v12000>(p);
+  }
+  return fn;
+}
+
+// bf16 tensor map.  dims/strides innermost first; strides (bytes) for dims 1..rank-1.
+static eas_status make_tmap(CUtensorMap* m, const void* base, int rank, const uint64_t* dims, const uint64_t* strides,
+                            const uint32_t* box, CUtensorMapSwizzle swz) {
+  PFN_cuTensorMapEncodeTiled_v12000 fn = get_encode_fn();
+  if (fn == nullptr) return fail(EAS_ERR_CUDA, "cuTensorMapEncodeTiled is not available from the driver");
+  cuuint64_t gdim[5], gstr[5];
+  cuuint32_t bx[5], es[5];
+  for (int i = 0; i < rank; ++i) { gdim[i] = dims[i]; bx[i] = box[i]; es[i] = 1; }
+  for (int i = 0; i + 1 < rank; ++i) gstr[i] = strides[i];
+  CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, rank, const_cast<void*>(base), gdim, gstr, bx, es,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return fail(EAS_ERR_CUDA, "cuTensorMapEncodeTiled failed with code %d", static_cast<int>(r));
+  return EAS_OK;
+}
+
+// W [N, K] row-major -> 2-D map, box 64 x 256
+static eas_status make_w_tmap(CUtensorMap* m, const void* w, int64_t N, int64_t K) {
+  const uint64_t dims[2] = {static_cast<uint64_t>(K), static_cast<uint64_t>(N)};
+  const uint64_t strides[1] = {static_cast<uint64_t>(K) * 2};
+  const uint32_t box[2] = {kBK, kBN};
+  return make_tmap(m, w, 2, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B);
+}
+// A as {run, phase, rows}: a plain [M, K] matrix is {K, 1, M}; a k=3 convolution over rows of width C with row
+// stride s is {C, s, rows/s} and the kernel walks taps as extra k-blocks
+static eas_status make_a_tmap(CUtensorMap* m, const void* a, int64_t run, int64_t row_elems, int conv_stride, int64_t rows) {
+  const uint64_t dims[3] = {static_cast<uint64_t>(run), static_cast<uint64_t>(conv_stride),
+                            static_cast<uint64_t>((rows + conv_stride - 1) / conv_stride)};
+  const uint64_t strides[2] = {static_cast<uint64_t>(row_elems) * 2, static_cast<uint64_t>(row_elems) * 2 * conv_stride};
+  const uint32_t box[3] = {kBK, 1, kBM};
+  return make_tmap(m, a, 3, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B);
+}
+
+// ------------------------------------------------------------------------------------ handle
+struct Linear {
+  const bf16* w = nullptr;   // [N, K] (possibly re-laid)
+  const bf16* b = nullptr;   // [N]
+  int N = 0, K = 0;
+  CUtensorMap tmap;
+};
+struct Layer {
+  const bf16 *n1g = nullptr, *n1b = nullptr, *n2g = nullptr, *n2b = nullptr;
+  Linear qkv, proj, fc1, fc2;
+};
+
+struct eas_encoder {
+  eas_arch_config cfg;
+  int sm_count = 0;
+  int hd = 0;
+  int embed_k = 0, embed_k_pad = 0;
+  Linear embed, conv1, conv2, head1, head2;
+  const bf16 *cls = nullptr, *pos = nullptr, *eng = nullptr, *enb = nullptr, *fng = nullptr, *fnb = nullptr, *hng = nullptr;
+  std::vector<Layer> layers;
+  int attn_impl = 0;
+  int last_launches = 0;
+  uint32_t* last_status = nullptr;
+};
+
+static size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+static eas_status check_cfg(const eas_arch_config* c) {
+  if (c == nullptr) return fail(EAS_ERR_INVALID_ARG, "arch config is null");
+  if (c->family < 0 || c->family > 2) return fail(EAS_ERR_INVALID_ARG, "unknown family %d", c->family);
+  if (c->n_layers < 0 || c->d_model <= 0 || c->n_heads <= 0 || c->d_mlp <= 0)
+    return fail(EAS_ERR_INVALID_ARG, "non-positive model dimension");
+  if (c->d_model % c->n_heads != 0) return fail(EAS_ERR_INVALID_ARG, "d_model %% n_heads != 0");
+  const int hd = c->d_model / c->n_heads;
+  if (hd != 64 && hd != 80) return fail(EAS_ERR_UNSUPPORTED, "head_dim %d (supported: 64, 80)", hd);
+  if (c->d_model % 128 != 0 || c->d_model > 2048) return fail(EAS_ERR_UNSUPPORTED, "d_model must be a multiple of 128, at most 2048");
+  if (c->d_mlp % 64 != 0) return fail(EAS_ERR_UNSUPPORTED, "d_mlp must be a multiple of 64");
+  if (c->norm != EAS_NORM_LAYERNORM && c->norm != EAS_NORM_RMSNORM) return fail(EAS_ERR_INVALID_ARG, "unknown norm");
+  if (c->mlp != EAS_MLP_GELU && c->mlp != EAS_MLP_SWIGLU) return fail(EAS_ERR_INVALID_ARG, "unknown mlp");
+  if (c->pos != EAS_POS_TABLE && c->pos != EAS_POS_ROPE_2D) return fail(EAS_ERR_INVALID_ARG, "unknown position scheme");
+  if (c->head < 0 || c->head > 2) return fail(EAS_ERR_INVALID_ARG, "unknown head");
+  if (c->in_channels <= 0 || c->patch <= 0 || c->temporal_patch <= 0) return fail(EAS_ERR_INVALID_ARG, "bad input geometry");
+  if (c->family == EAS_FAMILY_VIT_LEARNED && (c->pos != EAS_POS_TABLE || c->max_pos <= 0))
+    return fail(EAS_ERR_INVALID_ARG, "learned-position ViT needs a position table");
+  if (c->family == EAS_FAMILY_VIT_ROPE_MERGER && (c->pos != EAS_POS_ROPE_2D || c->head != EAS_HEAD_MERGER_2X2 || c->has_cls))
+    return fail(EAS_ERR_INVALID_ARG, "RoPE ViT needs 2-D rotary positions, the 2x2 merger and no CLS");
+  if (c->family == EAS_FAMILY_AUDIO_CONV && (c->pos != EAS_POS_TABLE || c->has_cls || c->in_channels % 64 != 0 || c->head != EAS_HEAD_NONE))
+    return fail(EAS_ERR_INVALID_ARG, "audio encoder needs a position table, mel bins %% 64 == 0, no CLS, no head");
+  if (c->pos == EAS_POS_ROPE_2D && (hd % 4 != 0 || c->rope_theta <= 1.0f)) return fail(EAS_ERR_INVALID_ARG, "bad rotary setup");
+  if (c->head != EAS_HEAD_NONE && (c->d_head_hidden <= 0 || c->d_head_hidden % 64 != 0 || c->d_out % 32 != 0))
+    return fail(EAS_ERR_UNSUPPORTED, "connector widths must be multiples of 64 (hidden) and 32 (out)");
+  if (c->head == EAS_HEAD_NONE && c->d_out != c->d_model) return fail(EAS_ERR_INVALID_ARG, "d_out must equal d_model without a head");
+  if (c->head == EAS_HEAD_MLP_PROJECTOR && c->final_norm) return fail(EAS_ERR_UNSUPPORTED, "projector after a final norm");
+  return EAS_OK;
+}
+
+static int embed_k_of(const eas_arch_config* c) { return c->in_channels * c->temporal_patch * c->patch * c->patch; }
+
+extern "C" size_t eas_encoder_weight_arena_bytes(const eas_arch_config* c) {
+  if (check_cfg(c) != EAS_OK) return 0;
+  size_t total = 1024;
+  const size_t d = c->d_model, I = c->d_mlp;
+  if (c->family != EAS_FAMILY_AUDIO_CONV) total += align_up(d * align_up(embed_k_of(c), 64) * 2, 1024);
+  if (c->pos == EAS_POS_ROPE_2D) total += c->n_layers * (align_up(3 * d * d * 2, 1024) + align_up(3 * d * 2, 1024));
+  if (c->mlp == EAS_MLP_SWIGLU) total += c->n_layers * (align_up(2 * I * d * 2, 1024) + align_up(2 * I * 2, 1024));
+  return total;
+}
+
+namespace {
+struct WeightIndex {
+  std::map<std::string, const eas_tensor*> by_name;
+  eas_status get(const std::string& name, std::initializer_list<int64_t> shape, const bf16** out) const {
+    auto it = by_name.find(name);
+    if (it == by_name.end()) return fail(EAS_ERR_INVALID_ARG, "weight '%s' is missing", name.c_str());
+    const eas_tensor* t = it->second;
+    if (t->dev_ptr == nullptr || (reinterpret_cast<uintptr_t>(t->dev_ptr) & 15) != 0)
+      return fail(EAS_ERR_INVALID_ARG, "weight '%s' has a null or unaligned pointer", name.c_str());
+    if (t->ndim != static_cast<int>(shape.size())) return fail(EAS_ERR_INVALID_ARG, "weight '%s' has rank %d", name.c_str(), t->ndim);
+    int i = 0;
+    for (int64_t s : shape) {
+      if (t->shape[i] != s)
+        return fail(EAS_ERR_INVALID_ARG, "weight '%s' dim %d is %lld, expected %lld", name.c_str(), i,
+                    static_cast<long long>(t->shape[i]), static_cast<long long>(s));
+      ++i;
+    }
+    *out = static_cast<const bf16*>(t->dev_ptr);
+    return EAS_OK;
+  }
+};
+
+struct Arena {
+  uint8_t* base; size_t size; size_t used = 0;
+  void* take(size_t bytes) {
+    const size_t off = align_up(used, 1024);
+    if (off + bytes > size) return nullptr;
+    used = off + bytes;
+    return base + off;
+  }
+};
+}  // namespace
+
+static eas_status relayout(bf16* dst, const bf16* src, const bf16* src2, long long rows, int k, int k_pad, int mode,
+                           int head_dim, long long rope_rows) {
+  RelayoutParams rp{src, src2, dst, rows, k, k_pad, mode, head_dim, rope_rows};
+  const long long total = rows * k_pad;
+  const int blocks = static_cast<int>(std::min<long long>((total + 255) / 256, 4096));
+  relayout_kernel<<<blocks, 256>>>(rp);
+  CUDA_TRY(cudaGetLastError());
+  return EAS_OK;
+}
+
+#define EAS_TRY(expr)            \
+  do {                           \
+    eas_status s_ = (expr);      \
+    if (s_ != EAS_OK) return s_; \
+  } while (0)
+
+static eas_status finish_linear(Linear& L) { return make_w_tmap(&L.tmap, L.w, L.N, L.K); }
+
+static eas_status set_kernel_attributes() {
+  CUDA_TRY(cudaFuncSetAttribute(gemm_kernel<ACT_NONE, OUT_BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmemBytes));
+  CUDA_TRY(cudaFuncSetAttribute(gemm_kernel<ACT_GELU, OUT_BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmemBytes));
+  CUDA_TRY(cudaFuncSetAttribute(gemm_kernel<ACT_SWIGLU, OUT_BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmemBytes));
+  CUDA_TRY(cudaFuncSetAttribute(gemm_kernel<ACT_NONE, OUT_F32>, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmemBytes));
+  CUDA_TRY(cudaFuncSetAttribute(gemm_kernel<ACT_GELU, OUT_F32>, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmemBytes));
+  return EAS_OK;
+}
+
+// shared memory requested by the light kernels: more than half an SM's capacity, so that a second CTA
+// can never be co-resident and a grid of B CTAs occupies B SMs
+constexpr int kOnePerSmSmem = 120 * 1024;
+
+static eas_status device_check(int* sm_count) {
+  int dev = 0;
+  CUDA_TRY(cudaGetDevice(&dev));
+  cudaDeviceProp prop;
+  CUDA_TRY(cudaGetDeviceProperties(&prop, dev));
+  if (prop.major != 10) return fail(EAS_ERR_ARCH, "device is compute capability %d.%d; this library is built for 10.x", prop.major, prop.minor);
+  *sm_count = prop.multiProcessorCount;
+  return EAS_OK;
+}
+
+extern "C" eas_status eas_encoder_create(const eas_arch_config* arch, const eas_weights* weights, eas_encoder** out) {
+  if (out == nullptr) return fail(EAS_ERR_INVALID_ARG, "out is null");
+  *out = nullptr;
+  EAS_TRY(check_cfg(arch));
+  if (weights == nullptr || weights->tensors == nullptr || weights->n_tensors <= 0)
+    return fail(EAS_ERR_INVALID_ARG, "weights are null or empty");
+  const size_t need = eas_encoder_weight_arena_bytes(arch);
+  if (weights->arena == nullptr || weights->arena_bytes < need)
+    return fail(EAS_ERR_WORKSPACE, "weight arena too small: %zu bytes given, %zu needed", weights->arena_bytes, need);
+  int sm_count = 0;
+  EAS_TRY(device_check(&sm_count));
+  EAS_TRY(set_kernel_attributes());
+
+  WeightIndex wi;
+  for (int i = 0; i < weights->n_tensors; ++i) {
+    if (weights->tensors[i].name == nullptr) return fail(EAS_ERR_INVALID_ARG, "tensor %d has no name", i);
+    wi.by_name[weights->tensors[i].name] = &weights->tensors[i];
+  }
+  eas_encoder* e = new eas_encoder();
+  std::unique_ptr<eas_encoder> guard(e);
+  e->cfg = *arch;
+  e->sm_count = sm_count;
+  const eas_arch_config& c = e->cfg;
+  const int d = c.d_model, I = c.d_mlp;
+  e->hd = d / c.n_heads;
+  const bool ln = c.norm == EAS_NORM_LAYERNORM;
+  Arena arena{static_cast<uint8_t*>(weights->arena), weights->arena_bytes};
+
+  if (c.family == EAS_FAMILY_AUDIO_CONV) {
+    EAS_TRY(wi.get("conv1.w", {d, 3, c.in_channels}, &e->conv1.w));
+    EAS_TRY(wi.get("conv1.b", {d}, &e->conv1.b));
+    e->conv1.N = d; e->conv1.K = 3 * c.in_channels;
+    EAS_TRY(finish_linear(e->conv1));
+    EAS_TRY(wi.get("conv2.w", {d, 3, d}, &e->conv2.w));
+    EAS_TRY(wi.get("conv2.b", {d}, &e->conv2.b));
+    e->conv2.N = d; e->conv2.K = 3 * d;
+    EAS_TRY(finish_linear(e->conv2));
+  } else {
+    e->embed_k = embed_k_of(&c);
+    e->embed_k_pad = static_cast<int>(align_up(e->embed_k, 64));
+    const bf16* w = nullptr;
+    EAS_TRY(wi.get("embed.w", {d, e->embed_k}, &w));
+    EAS_TRY(wi.get("embed.b", {d}, &e->embed.b));
+    bf16* dst = static_cast<bf16*>(arena.take(static_cast<size_t>(d) * e->embed_k_pad * 2));
+    if (dst == nullptr) return fail(EAS_ERR_WORKSPACE, "weight arena exhausted");
+    EAS_TRY(relayout(dst, w, nullptr, d, e->embed_k, e->embed_k_pad, 0, 0, 0));
+    e->embed.w = dst; e->embed.N = d; e->embed.K = e->embed_k_pad;
+    EAS_TRY(finish_linear(e->embed));
+  }
+  if (c.has_cls) EAS_TRY(wi.get("cls", {d}, &e->cls));
+  if (c.pos == EAS_POS_TABLE) EAS_TRY(wi.get("pos", {c.max_pos, d}, &e->pos));
+  if (c.embed_norm) {
+    EAS_TRY(wi.get("embed_norm.g", {d}, &e->eng));
+    if (ln) EAS_TRY(wi.get("embed_norm.b", {d}, &e->enb));
+  }
+  e->layers.resize(c.n_layers);
+  for (int i = 0; i < c.n_layers; ++i) {
+    Layer& L = e->layers[i];
+    const std::string p = "blk" + std::to_string(i) + ".";
+    EAS_TRY(wi.get(p + "norm1.g", {d}, &L.n1g));
+    if (ln) EAS_TRY(wi.get(p + "norm1.b", {d}, &L.n1b));
+    EAS_TRY(wi.get(p + "norm2.g", {d}, &L.n2g));
+    if (ln) EAS_TRY(wi.get(p + "norm2.b", {d}, &L.n2b));
+    const bf16 *qw = nullptr, *qb = nullptr;
+    EAS_TRY(wi.get(p + "qkv.w", {3 * d, d}, &qw));
+    EAS_TRY(wi.get(p + "qkv.b", {3 * d}, &qb));
+    if (c.pos == EAS_POS_ROPE_2D) {
+      // rows of every Q and K head re-ordered so that the two halves of a rotary pair are adjacent
+      bf16* w2 = static_cast<bf16*>(arena.take(static_cast<size_t>(3) * d * d * 2));
+      bf16* b2 = static_cast<bf16*>(arena.take(static_cast<size_t>(3) * d * 2));
+      if (w2 == nullptr || b2 == nullptr) return fail(EAS_ERR_WORKSPACE, "weight arena exhausted");
+      EAS_TRY(relayout(w2, qw, nullptr, 3LL * d, d, d, 1, e->hd, 2LL * d));
+      EAS_TRY(relayout(b2, qb, nullptr, 3LL * d, 1, 1, 1, e->hd, 2LL * d));
+      qw = w2; qb = b2;
+    }
+    L.qkv.w = qw; L.qkv.b = qb; L.qkv.N = 3 * d; L.qkv.K = d;
+    EAS_TRY(finish_linear(L.qkv));
+    EAS_TRY(wi.get(p + "proj.w", {d, d}, &L.proj.w));
+    EAS_TRY(wi.get(p + "proj.b", {d}, &L.proj.b));
+    L.proj.N = d; L.proj.K = d;
+    EAS_TRY(finish_linear(L.proj));
+    if (c.mlp == EAS_MLP_SWIGLU) {
+      const bf16 *gw, *gb, *uw, *ub;
+      EAS_TRY(wi.get(p + "gate.w", {I, d}, &gw));
+      EAS_TRY(wi.get(p + "gate.b", {I}, &gb));
+      EAS_TRY(wi.get(p + "up.w", {I, d}, &uw));
+      EAS_TRY(wi.get(p + "up.b", {I}, &ub));
+      bf16* w2 = static_cast<bf16*>(arena.take(static_cast<size_t>(2) * I * d * 2));
+      bf16* b2 = static_cast<bf16*>(arena.take(static_cast<size_t>(2) * I * 2));
+      if (w2 == nullptr || b2 == nullptr) return fail(EAS_ERR_WORKSPACE, "weight arena exhausted");
+      EAS_TRY(relayout(w2, gw, uw, 2LL * I, d, d, 2, 0, 0));
+      EAS_TRY(relayout(b2, gb, ub, 2LL * I, 1, 1, 2, 0, 0));
+      L.fc1.w = w2; L.fc1.b = b2; L.fc1.N = 2 * I; L.fc1.K = d;
+    } else {
+      EAS_TRY(wi.get(p + "fc1.w", {I, d}, &L.fc1.w));
+      EAS_TRY(wi.get(p + "fc1.b", {I}, &L.fc1.b));
+      L.fc1.N = I; L.fc1.K = d;
+    }
+    EAS_TRY(finish_linear(L.fc1));
+    EAS_TRY(wi.get(p + "fc2.w", {d, I}, &L.fc2.w));
+    EAS_TRY(wi.get(p + "fc2.b", {d}, &L.fc2.b));
+    L.fc2.N = d; L.fc2.K = I;
+    EAS_TRY(finish_linear(L.fc2));
+  }
+  if (c.final_norm) {
+    EAS_TRY(wi.get("final_norm.g", {d}, &e->fng));
+    if (ln) EAS_TRY(wi.get("final_norm.b", {d}, &e->fnb));
+  }
+  if (c.head != EAS_HEAD_NONE) {
+    const int kin = c.head == EAS_HEAD_MERGER_2X2 ? 4 * d : d;
+    if (c.head == EAS_HEAD_MERGER_2X2) EAS_TRY(wi.get("head.norm.g", {d}, &e->hng));
+    EAS_TRY(wi.get("head.fc1.w", {c.d_head_hidden, kin}, &e->head1.w));
+    EAS_TRY(wi.get("head.fc1.b", {c.d_head_hidden}, &e->head1.b));
+    e->head1.N = c.d_head_hidden; e->head1.K = kin;
+    EAS_TRY(finish_linear(e->head1));
+    EAS_TRY(wi.get("head.fc2.w", {c.d_out, c.d_head_hidden}, &e->head2.w));
+    EAS_TRY(wi.get("head.fc2.b", {c.d_out}, &e->head2.b));
+    e->head2.N = c.d_out; e->head2.K = c.d_head_hidden;
+    EAS_TRY(finish_linear(e->head2));
+  }
+  CUDA_TRY(cudaDeviceSynchronize());   // re-layout kernels ran on the default stream
+  *out = guard.release();
+  return EAS_OK;
+}
+
+extern "C" void eas_encoder_destroy(eas_encoder* enc) { delete enc; }
+
+extern "C" eas_status eas_encoder_set_attention_impl(eas_encoder* enc, int32_t impl) {
+  if (enc == nullptr || impl < 0 || impl > 1) return fail(EAS_ERR_INVALID_ARG, "bad attention impl");
+  enc->attn_impl = impl;
+  return EAS_OK;
+}
+
+extern "C" int32_t eas_encoder_last_launch_count(const eas_encoder* enc) { return enc ? enc->last_launches : 0; }
+
+// ------------------------------------------------------------------------------------ workspace plan
+namespace {
+struct Plan {
+  size_t status, x, n, qkv, o, a, embed_a, row_map, pos_idx, head_src, rope, mel_pad, h1_pad, conv1_map, total;
+  int64_t T, embed_rows, padded_rows, out_rows;
+};
+}  // namespace
+
+static Plan make_plan(const eas_encoder* e, int64_t T, int n_items) {
+  const eas_arch_config& c = e->cfg;
+  Plan p{};
+  p.T = T;
+  size_t off = 0;
+  auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 1024); return o; };
+  const size_t d = c.d_model;
+  const bool audio = c.family == EAS_FAMILY_AUDIO_CONV;
+  p.padded_rows = audio ? 2 * T + 2 * n_items : 0;
+  p.embed_rows = audio ? T + n_items : T - (c.has_cls ? n_items : 0);
+  p.out_rows = c.head == EAS_HEAD_MLP_PROJECTOR ? T - (c.has_cls ? n_items : 0) : (c.head == EAS_HEAD_MERGER_2X2 ? T / 4 : T);
+  p.status = take(1024);
+  p.x = take(T * d * 4);
+  p.n = take(T * d * 2);
+  p.qkv = take(T * 3 * d * 2);
+  p.o = take(T * d * 2);
+  const size_t a_elems = std::max<size_t>(T * static_cast<size_t>(c.d_mlp), static_cast<size_t>(p.out_rows) * std::max(c.d_head_hidden, 0));
+  p.a = take(a_elems * 2);
+  p.embed_a = take(audio ? 0 : static_cast<size_t>(p.embed_rows) * e->embed_k_pad * 2);
+  p.row_map = take(static_cast<size_t>(p.embed_rows) * 4);
+  p.pos_idx = take(static_cast<size_t>(p.embed_rows) * 4);
+  p.head_src = take(static_cast<size_t>(T) * 4);
+  p.rope = take(c.pos == EAS_POS_ROPE_2D ? static_cast<size_t>(T) * (e->hd / 2) * 8 : 0);
+  p.mel_pad = take(static_cast<size_t>(p.padded_rows) * c.in_channels * 2);
+  p.h1_pad = take(static_cast<size_t>(p.padded_rows) * d * 2);
+  p.conv1_map = take(static_cast<size_t>(p.padded_rows) * 4);
+  p.total = off;
+  return p;
+}
+
+extern "C" size_t eas_encoder_workspace_bytes(const eas_encoder* enc, int64_t total_tokens, int32_t n_items, int32_t /*max_seqlen*/) {
+  if (enc == nullptr || total_tokens <= 0 || n_items <= 0) return 0;
+  return make_plan(enc, total_tokens, n_items).total;
+}
+
+static int64_t out_rows_of(const eas_encoder* e, int64_t S) {
+  if (e->cfg.head == EAS_HEAD_MLP_PROJECTOR) return S - (e->cfg.has_cls ? 1 : 0);
+  if (e->cfg.head == EAS_HEAD_MERGER_2X2) return S / 4;
+  return S;
+}
+
+extern "C" int64_t eas_encoder_out_rows(const eas_encoder* enc, const int32_t* cu, int32_t n_items) {
+  if (enc == nullptr || cu == nullptr || n_items <= 0) return -1;
+  int64_t r = 0;
+  for (int i = 0; i < n_items; ++i) r += out_rows_of(enc, cu[i + 1] - cu[i]);
+  return r;
+}
+
+// ------------------------------------------------------------------------------------ launch helpers
+namespace {
+struct GemmCall {
+  const void* A = nullptr;   // bf16
+  int64_t a_run = 0;         // K per tap (elements)
+  int64_t a_row_elems = 0;   // elements between consecutive rows of A
+  int conv_stride = 1;       // 1: plain GEMM
+  int taps = 1;
+  int64_t a_rows = 0;        // rows addressable in A
+  int M = 0;                 // rows walked
+  const Linear* lin = nullptr;
+  int act = ACT_NONE;
+  int out_fp32 = 0;
+  void* out = nullptr;
+  int64_t ldo = 0;
+  const float* resid = nullptr;
+  const int* row_map = nullptr;
+  const int* pos_idx = nullptr;
+  const bf16* pos = nullptr;
+  const float2* rope_cs = nullptr;
+  int rope_pairs = 0, rope_ncols = 0, head_dim = 0;
+};
+}  // namespace
+
+static eas_status launch_gemm(const GemmCall& g, int budget, cudaStream_t stream, uint32_t* status) {
+  const Linear& L = *g.lin;
+  if (g.M <= 0) return EAS_OK;
+  if (L.N % 32 != 0 || g.a_run % kBK != 0) return fail(EAS_ERR_UNSUPPORTED, "GEMM needs N %% 32 == 0 and K %% 64 == 0 (N=%d, K=%lld)", L.N, static_cast<long long>(g.a_run));
+  GemmParams p{};
+  EAS_TRY(make_a_tmap(&p.tma_a, g.A, g.a_run, g.a_row_elems, g.conv_stride, g.a_rows));
+  p.tma_b = L.tmap;
+  p.M = g.M; p.N = L.N;
+  p.kb_per_tap = static_cast<int>(g.a_run / kBK);
+  p.k_blocks = p.kb_per_tap * g.taps;
+  p.conv_stride = g.conv_stride;
+  p.m_blocks = (g.M + kBM - 1) / kBM;
+  p.n_blocks = (L.N + kBN - 1) / kBN;
+  p.bias = L.b;
+  p.out = g.out; p.ldo = g.ldo; p.resid = g.resid;
+  p.row_map = g.row_map; p.pos_idx = g.pos_idx; p.pos = g.pos;
+  p.rope_cs = g.rope_cs; p.rope_pairs = g.rope_pairs; p.rope_ncols = g.rope_ncols; p.head_dim = g.head_dim > 0 ? g.head_dim : 64;
+  p.status = status;
+  const int tiles = p.m_blocks * p.n_blocks;
+  const int grid = std::min(budget, tiles);
+  void (*kern)(GemmParams) = nullptr;
+  if (g.act == ACT_NONE && !g.out_fp32) kern = gemm_kernel<ACT_NONE, OUT_BF16>;
+  else if (g.act == ACT_GELU && !g.out_fp32) kern = gemm_kernel<ACT_GELU, OUT_BF16>;
+  else if (g.act == ACT_SWIGLU && !g.out_fp32) kern = gemm_kernel<ACT_SWIGLU, OUT_BF16>;
+  else if (g.act == ACT_NONE && g.out_fp32) kern = gemm_kernel<ACT_NONE, OUT_F32>;
+  else if (g.act == ACT_GELU && g.out_fp32) kern = gemm_kernel<ACT_GELU, OUT_F32>;
+  else return fail(EAS_ERR_UNSUPPORTED, "no GEMM epilogue for act=%d out_fp32=%d", g.act, g.out_fp32);
+  kern<<<grid, kGemmThreads, kGemmSmemBytes, stream>>>(p);
+  CUDA_TRY(cudaGetLastError());
+  return EAS_OK;
+}
+
+template <int KIND, bool F32>
+static eas_status launch_norm_nv(const NormParams& p, int budget, cudaStream_t stream) {
+  const int nv = p.d / 128;
+#define EAS_NORM_CASE(NV_)                                                                                         \
+  case NV_: {                                                                                                      \
+    static bool attr_set = false;                                                                                  \
+    if (!attr_set) {                                                                                               \
+      CUDA_TRY(cudaFuncSetAttribute(norm_kernel<NV_, KIND, F32>, cudaFuncAttributeMaxDynamicSharedMemorySize, kOnePerSmSmem)); \
+      attr_set = true;                                                                                             \
+    }                                                                                                              \
+    norm_kernel<NV_, KIND, F32><<<std::min(budget, (p.rows + 15) / 16), 512, kOnePerSmSmem, stream>>>(p);          \
+    break;                                                                                                         \
+  }
+  switch (nv) {
+    EAS_NORM_CASE(1) EAS_NORM_CASE(2) EAS_NORM_CASE(3) EAS_NORM_CASE(4) EAS_NORM_CASE(5) EAS_NORM_CASE(6)
+    EAS_NORM_CASE(7) EAS_NORM_CASE(8) EAS_NORM_CASE(9) EAS_NORM_CASE(10) EAS_NORM_CASE(11) EAS_NORM_CASE(12)
+    EAS_NORM_CASE(13) EAS_NORM_CASE(14) EAS_NORM_CASE(15) EAS_NORM_CASE(16)
+    default: return fail(EAS_ERR_UNSUPPORTED, "norm width %d", p.d);
+  }
+#undef EAS_NORM_CASE
+  CUDA_TRY(cudaGetLastError());
+  return EAS_OK;
+}
+
+static eas_status launch_norm(int kind, bool out_fp32, const NormParams& p, int budget, cudaStream_t stream) {
+  if (p.rows <= 0) return EAS_OK;
+  if (p.d % 128 != 0 || p.d > 2048) return fail(EAS_ERR_UNSUPPORTED, "norm width %d (need a multiple of 128, at most 2048)", p.d);
+  if (kind == NORM_LN) return out_fp32 ? launch_norm_nv<NORM_LN, true>(p, budget, stream) : launch_norm_nv<NORM_LN, false>(p, budget, stream);
+  if (kind == NORM_RMS) return out_fp32 ? launch_norm_nv<NORM_RMS, true>(p, budget, stream) : launch_norm_nv<NORM_RMS, false>(p, budget, stream);
+  if (kind == NORM_CAST) return out_fp32 ? fail(EAS_ERR_UNSUPPORTED, "fp32 cast") : launch_norm_nv<NORM_CAST, false>(p, budget, stream);
+  return fail(EAS_ERR_INVALID_ARG, "unknown norm kind %d", kind);
+}
+
+static eas_status launch_attention(const bf16* qkv, bf16* out, const int32_t* cu, int n_items, int H, int hd, int budget,
+                                   cudaStream_t stream, int /*impl*/, uint32_t* /*status*/) {
+  AttnParams ap{};
+  const int d = H * hd;
+  ap.qkv = qkv; ap.out = out; ap.ld = 3LL * d; ap.ldo = d; ap.d_model = d; ap.n_heads = H;
+  ap.scale_log2 = static_cast<float>(1.4426950408889634 / std::sqrt(static_cast<double>(hd)));
+  ap.n_items = n_items;
+  // schedule order: longest items first (stable), so the tail of the static round-robin is short work
+  std::vector<int> order(n_items);
+  for (int i = 0; i < n_items; ++i) order[i] = i;
+  std::stable_sort(order.begin(), order.end(), [&](int a, int b) { return (cu[a + 1] - cu[a]) > (cu[b + 1] - cu[b]); });
+  int units = 0;
+  for (int k = 0; k < n_items; ++k) {
+    const int i = order[k];
+    ap.item_start[k] = cu[i];
+    ap.item_len[k] = cu[i + 1] - cu[i];
+    ap.unit_prefix[k] = units;
+    units += ((ap.item_len[k] + kAttnBQ - 1) / kAttnBQ) * H;
+  }
+  ap.unit_prefix[n_items] = units;
+  ap.total_units = units;
+  if (units == 0) return EAS_OK;
+  const int grid = std::min(budget, units);
+  static bool attr_set = false;
+  if (!attr_set) {
+    CUDA_TRY(cudaFuncSetAttribute(attn_mma_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, kOnePerSmSmem));
+    CUDA_TRY(cudaFuncSetAttribute(attn_mma_kernel<80>, cudaFuncAttributeMaxDynamicSharedMemorySize, kOnePerSmSmem));
+    attr_set = true;
+  }
+  static_assert(attn_mma_smem_bytes<80>() <= kOnePerSmSmem, "attention tile does not fit");
+  if (hd == 64) attn_mma_kernel<64><<<grid, kAttnThreads, kOnePerSmSmem, stream>>>(ap);
+  else if (hd == 80) attn_mma_kernel<80><<<grid, kAttnThreads, kOnePerSmSmem, stream>>>(ap);
+  else return fail(EAS_ERR_UNSUPPORTED, "head_dim %d", hd);
+  CUDA_TRY(cudaGetLastError());
+  return EAS_OK;
+}
+
+// ------------------------------------------------------------------------------------ the forward pass
+extern "C" eas_status eas_encode_microbatch(eas_encoder* e, const eas_packed_inputs* in, const int32_t* cu_dev,
+                                            int32_t sm_budget, void* stream_v, void* out_embeddings) {
+  if (e == nullptr || in == nullptr) return fail(EAS_ERR_INVALID_ARG, "encoder or inputs are null");
+  if (in->data == nullptr || in->item_shape == nullptr || in->item_offset == nullptr || in->cu_seqlens_host == nullptr ||
+      in->workspace == nullptr || cu_dev == nullptr || out_embeddings == nullptr)
+    return fail(EAS_ERR_INVALID_ARG, "a required pointer is null");
+  const int n = in->n_items;
+  if (n < 1 || n > EAS_MAX_ITEMS) return fail(EAS_ERR_INVALID_ARG, "n_items %d outside 1..%d", n, static_cast<int>(EAS_MAX_ITEMS));
+  if (sm_budget < 0 || sm_budget > e->sm_count) return fail(EAS_ERR_INVALID_ARG, "sm_budget %d outside 0..%d", sm_budget, e->sm_count);
+  if ((reinterpret_cast<uintptr_t>(in->workspace) & 1023) != 0) return fail(EAS_ERR_INVALID_ARG, "workspace is not 1024-byte aligned");
+  if ((reinterpret_cast<uintptr_t>(in->data) & 15) != 0 || (reinterpret_cast<uintptr_t>(out_embeddings) & 15) != 0)
+    return fail(EAS_ERR_INVALID_ARG, "data / out_embeddings must be 16-byte aligned");
+  const int budget = sm_budget == 0 ? e->sm_count : sm_budget;
+  const eas_arch_config& c = e->cfg;
+  const int32_t* cu = in->cu_seqlens_host;
+  const int d = c.d_model;
+  const bool audio = c.family == EAS_FAMILY_AUDIO_CONV;
+  if (cu[0] != 0) return fail(EAS_ERR_INVALID_ARG, "cu_seqlens must start at 0");
+
+  ItemTable items{};
+  items.n_items = n;
+  int aux = 0;
+  for (int i = 0; i < n; ++i) {
+    const int f = in->item_shape[3 * i], h = in->item_shape[3 * i + 1], w = in->item_shape[3 * i + 2];
+    const int S = cu[i + 1] - cu[i];
+    if (S <= 0) return fail(EAS_ERR_INVALID_ARG, "cu_seqlens is not strictly increasing at item %d", i);
+    if (f <= 0 || h <= 0 || w <= 0 || in->item_offset[i] < 0) return fail(EAS_ERR_INVALID_ARG, "item %d has a non-positive shape or negative offset", i);
+    int expect;
+    items.tok_start[i] = cu[i];
+    items.aux_start[i] = aux;
+    items.frames[i] = f; items.height[i] = h; items.width[i] = w;
+    items.offset[i] = in->item_offset[i];
+    if (audio) {
+      if (h != c.in_channels || w != 1) return fail(EAS_ERR_INVALID_ARG, "audio item %d must be (frames, %d, 1)", i, c.in_channels);
+      if (f % 2 != 0) return fail(EAS_ERR_INVALID_ARG, "audio item %d has an odd frame count", i);
+      if ((in->item_offset[i] * 2) % 16 != 0) return fail(EAS_ERR_INVALID_ARG, "item %d offset is not 16-byte aligned", i);
+      expect = f / 2;
+      aux += f + 2;
+    } else {
+      const int unit = c.patch * (c.head == EAS_HEAD_MERGER_2X2 ? 2 : 1);
+      if (h % unit != 0 || w % unit != 0) return fail(EAS_ERR_INVALID_ARG, "item %d: height/width must be multiples of %d", i, unit);
+      if (f % c.temporal_patch != 0) return fail(EAS_ERR_INVALID_ARG, "item %d: frames must be a multiple of %d", i, c.temporal_patch);
+      if (c.temporal_patch == 1 && f != 1) return fail(EAS_ERR_INVALID_ARG, "item %d: an image encoder takes one frame", i);
+      const int patches = (f / c.temporal_patch) * (h / c.patch) * (w / c.patch);
+      expect = patches + (c.has_cls ? 1 : 0);
+      aux += patches;
+    }
+    if (S != expect) return fail(EAS_ERR_INVALID_ARG, "item %d: cu_seqlens says %d tokens, its shape gives %d", i, S, expect);
+    if (c.pos == EAS_POS_TABLE && S > c.max_pos) return fail(EAS_ERR_INVALID_ARG, "item %d has %d tokens, position table has %d rows", i, S, c.max_pos);
+  }
+  items.tok_start[n] = cu[n];
+  items.aux_start[n] = aux;
+  const int64_t T = cu[n];
+  const Plan pl = make_plan(e, T, n);
+  if (in->workspace_bytes < pl.total) return fail(EAS_ERR_WORKSPACE, "workspace too small: %zu bytes given, %zu needed", in->workspace_bytes, pl.total);
+
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+  uint8_t* ws = static_cast<uint8_t*>(in->workspace);
+  uint32_t* status = reinterpret_cast<uint32_t*>(ws + pl.status);
+  float* x = reinterpret_cast<float*>(ws + pl.x);
+  bf16* nbuf = reinterpret_cast<bf16*>(ws + pl.n);
+  bf16* qkv = reinterpret_cast<bf16*>(ws + pl.qkv);
+  bf16* obuf = reinterpret_cast<bf16*>(ws + pl.o);
+  bf16* abuf = reinterpret_cast<bf16*>(ws + pl.a);
+  bf16* embed_a = reinterpret_cast<bf16*>(ws + pl.embed_a);
+  int* row_map = reinterpret_cast<int*>(ws + pl.row_map);
+  int* pos_idx = reinterpret_cast<int*>(ws + pl.pos_idx);
+  int* head_src = reinterpret_cast<int*>(ws + pl.head_src);
+  float2* rope = reinterpret_cast<float2*>(ws + pl.rope);
+  bf16* mel_pad = reinterpret_cast<bf16*>(ws + pl.mel_pad);
+  bf16* h1_pad = reinterpret_cast<bf16*>(ws + pl.h1_pad);
+  int* conv1_map = reinterpret_cast<int*>(ws + pl.conv1_map);
+  int launches = 0;
+  e->last_status = status;
+
+  CUDA_TRY(cudaMemsetAsync(status, 0, 16, stream));
+
+  // ---- tables: row maps, rotary (cos, sin), CLS rows
+  {
+    PrepParams pp{};
+    pp.items = items;
+    pp.family = c.family; pp.has_cls = c.has_cls; pp.patch = c.patch; pp.d_model = d;
+    pp.total_tokens = static_cast<int>(T); pp.n_embed_rows = static_cast<int>(pl.embed_rows);
+    pp.rope_pairs = e->hd / 2; pp.rope_theta = c.rope_theta;
+    pp.cu_seqlens_dev = cu_dev;
+    pp.embed_row_map = row_map; pp.embed_pos_idx = pos_idx;
+    pp.head_src_rows = c.head == EAS_HEAD_MLP_PROJECTOR ? head_src : nullptr;
+    pp.rope_cs = rope; pp.x = x; pp.cls = e->cls; pp.pos = e->pos;
+    pp.conv1_row_map = conv1_map; pp.n_conv1_rows = static_cast<int>(pl.padded_rows);
+    pp.status = status;
+    prep_kernel<<<budget, 256, 0, stream>>>(pp);
+    CUDA_TRY(cudaGetLastError());
+    ++launches;
+  }
+
+  // ---- embedding
+  const int ln_kind = c.norm == EAS_NORM_LAYERNORM ? NORM_LN : NORM_RMS;
+  if (audio) {
+    AudioStageParams sp{};
+    sp.data = static_cast<const bf16*>(in->data); sp.mel_pad = mel_pad; sp.h1_pad = h1_pad;
+    sp.n_mel = c.in_channels; sp.d_model = d; sp.padded_rows = static_cast<int>(pl.padded_rows); sp.items = items;
+    static bool attr_set = false;
+    if (!attr_set) { CUDA_TRY(cudaFuncSetAttribute(audio_stage_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kOnePerSmSmem)); attr_set = true; }
+    audio_stage_kernel<<<budget, 512, kOnePerSmSmem, stream>>>(sp);
+    CUDA_TRY(cudaGetLastError());
+    ++launches;
+    GemmCall g1;   // conv1 (k=3, stride 1) + GELU -> padded h1
+    g1.A = mel_pad; g1.a_run = c.in_channels; g1.a_row_elems = c.in_channels; g1.conv_stride = 1; g1.taps = 3;
+    g1.a_rows = pl.padded_rows; g1.M = static_cast<int>(pl.padded_rows); g1.lin = &e->conv1; g1.act = ACT_GELU;
+    g1.out = h1_pad; g1.ldo = d; g1.row_map = conv1_map;
+    EAS_TRY(launch_gemm(g1, budget, stream, status)); ++launches;
+    GemmCall g2;   // conv2 (k=3, stride 2) + GELU + position table -> residual stream
+    g2.A = h1_pad; g2.a_run = d; g2.a_row_elems = d; g2.conv_stride = 2; g2.taps = 3;
+    g2.a_rows = pl.padded_rows; g2.M = static_cast<int>(pl.embed_rows); g2.lin = &e->conv2; g2.act = ACT_GELU; g2.out_fp32 = 1;
+    g2.out = x; g2.ldo = d; g2.row_map = row_map; g2.pos_idx = pos_idx; g2.pos = e->pos;
+    EAS_TRY(launch_gemm(g2, budget, stream, status)); ++launches;
+  } else {
+    Im2colParams ip{};
+    ip.data = static_cast<const bf16*>(in->data); ip.a = embed_a;
+    ip.n_patches = static_cast<int>(pl.embed_rows); ip.k = e->embed_k; ip.k_pad = e->embed_k_pad;
+    ip.channels = c.in_channels; ip.patch = c.patch; ip.tpatch = c.temporal_patch;
+    ip.merge_order = c.family == EAS_FAMILY_VIT_ROPE_MERGER ? 1 : 0;
+    ip.items = items;
+    static bool attr_set = false;
+    if (!attr_set) { CUDA_TRY(cudaFuncSetAttribute(im2col_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kOnePerSmSmem)); attr_set = true; }
+    im2col_kernel<<<budget, 512, kOnePerSmSmem, stream>>>(ip);
+    CUDA_TRY(cudaGetLastError());
+    ++launches;
+    GemmCall g;
+    g.A = embed_a; g.a_run = e->embed_k_pad; g.a_row_elems = e->embed_k_pad; g.a_rows = pl.embed_rows; g.M = static_cast<int>(pl.embed_rows);
+    g.lin = &e->embed; g.out_fp32 = 1; g.out = x; g.ldo = d; g.row_map = row_map;
+    if (c.pos == EAS_POS_TABLE) { g.pos_idx = pos_idx; g.pos = e->pos; }
+    EAS_TRY(launch_gemm(g, budget, stream, status)); ++launches;
+  }
+  if (c.embed_norm) {
+    NormParams np{x, x, e->eng, e->enb, nullptr, static_cast<int>(T), d, c.norm_eps};
+    EAS_TRY(launch_norm(ln_kind, true, np, budget, stream)); ++launches;
+  }
+
+  // ---- transformer blocks
+  for (int li = 0; li < c.n_layers; ++li) {
+    const Layer& L = e->layers[li];
+    {
+      NormParams np{x, nbuf, L.n1g, L.n1b, nullptr, static_cast<int>(T), d, c.norm_eps};
+      EAS_TRY(launch_norm(ln_kind, false, np, budget, stream)); ++launches;
+    }
+    {
+      GemmCall g;
+      g.A = nbuf; g.a_run = d; g.a_row_elems = d; g.a_rows = T; g.M = static_cast<int>(T); g.lin = &L.qkv;
+      g.out = qkv; g.ldo = 3LL * d;
+      if (c.pos == EAS_POS_ROPE_2D) { g.rope_cs = rope; g.rope_pairs = e->hd / 2; g.rope_ncols = 2 * d; g.head_dim = e->hd; }
+      EAS_TRY(launch_gemm(g, budget, stream, status)); ++launches;
+    }
+    EAS_TRY(launch_attention(qkv, obuf, cu, n, c.n_heads, e->hd, budget, stream, e->attn_impl, status)); ++launches;
+    {
+      GemmCall g;
+      g.A = obuf; g.a_run = d; g.a_row_elems = d; g.a_rows = T; g.M = static_cast<int>(T); g.lin = &L.proj;
+      g.out_fp32 = 1; g.out = x; g.ldo = d; g.resid = x;
+      EAS_TRY(launch_gemm(g, budget, stream, status)); ++launches;
+    }
+    {
+      NormParams np{x, nbuf, L.n2g, L.n2b, nullptr, static_cast<int>(T), d, c.norm_eps};
+      EAS_TRY(launch_norm(ln_kind, false, np, budget, stream)); ++launches;
+    }
+    {
+      GemmCall g;
+      g.A = nbuf; g.a_run = d; g.a_row_elems = d; g.a_rows = T; g.M = static_cast<int>(T); g.lin = &L.fc1;
+      g.act = c.mlp == EAS_MLP_SWIGLU ? ACT_SWIGLU : ACT_GELU;
+      g.out = abuf; g.ldo = c.d_mlp;
+      EAS_TRY(launch_gemm(g, budget, stream, status)); ++launches;
+    }
+    {
+      GemmCall g;
+      g.A = abuf; g.a_run = c.d_mlp; g.a_row_elems = c.d_mlp; g.a_rows = T; g.M = static_cast<int>(T); g.lin = &L.fc2;
+      g.out_fp32 = 1; g.out = x; g.ldo = d; g.resid = x;
+      EAS_TRY(launch_gemm(g, budget, stream, status)); ++launches;
+    }
+  }
+
+  // ---- connector
+  if (c.head == EAS_HEAD_NONE) {
+    if (c.final_norm) {
+      NormParams np{x, out_embeddings, e->fng, e->fnb, nullptr, static_cast<int>(T), d, c.norm_eps};
+      EAS_TRY(launch_norm(ln_kind, false, np, budget, stream)); ++launches;
+    } else {
+      NormParams np{x, out_embeddings, nullptr, nullptr, nullptr, static_cast<int>(T), d, c.norm_eps};
+      EAS_TRY(launch_norm(NORM_CAST, false, np, budget, stream)); ++launches;
+    }
+  } else {
+    int64_t rows_in;   // rows of the connector's first GEMM
+    int64_t k_in;
+    if (c.head == EAS_HEAD_MLP_PROJECTOR) {
+      rows_in = pl.out_rows; k_in = d;
+      NormParams np{x, nbuf, nullptr, nullptr, c.has_cls ? head_src : nullptr, static_cast<int>(rows_in), d, c.norm_eps};
+      EAS_TRY(launch_norm(NORM_CAST, false, np, budget, stream)); ++launches;
+    } else {
+      // RMSNorm per token; four consecutive tokens (one 2x2 group) then form one row of width 4d
+      rows_in = T / 4; k_in = 4LL * d;
+      NormParams np{x, nbuf, e->hng, nullptr, nullptr, static_cast<int>(T), d, c.norm_eps};
+      EAS_TRY(launch_norm(NORM_RMS, false, np, budget, stream)); ++launches;
+    }
+    GemmCall g1;
+    g1.A = nbuf; g1.a_run = k_in; g1.a_row_elems = k_in; g1.a_rows = rows_in; g1.M = static_cast<int>(rows_in); g1.lin = &e->head1;
+    g1.act = ACT_GELU; g1.out = abuf; g1.ldo = c.d_head_hidden;
+    EAS_TRY(launch_gemm(g1, budget, stream, status)); ++launches;
+    GemmCall g2;
+    g2.A = abuf; g2.a_run = c.d_head_hidden; g2.a_row_elems = c.d_head_hidden; g2.a_rows = rows_in; g2.M = static_cast<int>(rows_in); g2.lin = &e->head2;
+    g2.out = out_embeddings; g2.ldo = c.d_out;
+    EAS_TRY(launch_gemm(g2, budget, stream, status)); ++launches;
+  }
+  e->last_launches = launches;
+  return EAS_OK;
+}
+
+extern "C" eas_status eas_encoder_status(eas_encoder* e, void* stream_v) {
+  if (e == nullptr) return fail(EAS_ERR_INVALID_ARG, "encoder is null");
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+  CUDA_TRY(cudaStreamSynchronize(stream));
+  if (e->last_status == nullptr) return EAS_OK;
+  uint32_t v = 0;
+  CUDA_TRY(cudaMemcpy(&v, e->last_status, 4, cudaMemcpyDeviceToHost));
+  if (v != DEV_OK) CUDA_TRY(cudaMemset(e->last_status, 0, 4));
+  if (v == DEV_ERR_WAIT_TIMEOUT) return fail(EAS_ERR_DEVICE_TIMEOUT, "a bounded device-side wait expired");
+  if (v == DEV_ERR_CU_SEQLENS_MISMATCH) return fail(EAS_ERR_DEVICE_CHECK, "device cu_seqlens differs from cu_seqlens_host");
+  if (v != DEV_OK) return fail(EAS_ERR_DEVICE_CHECK, "device status %u", v);
+  return EAS_OK;
+}
+
+// ------------------------------------------------------------------------------------ single-kernel entry points
+static eas_status resolve_budget(int32_t sm_budget, int* budget) {
+  int sm_count = 0;
+  EAS_TRY(device_check(&sm_count));
+  if (sm_budget < 0 || sm_budget > sm_count) return fail(EAS_ERR_INVALID_ARG, "sm_budget %d outside 0..%d", sm_budget, sm_count);
+  *budget = sm_budget == 0 ? sm_count : sm_budget;
+  return EAS_OK;
+}
+
+extern "C" eas_status eas_kernel_gemm(const void* A, const void* W, const void* bias, void* out, const float* resid,
+                                      int32_t M, int32_t N, int32_t K, int32_t act, int32_t out_fp32, int32_t sm_budget,
+                                      void* stream, uint32_t* status_dev) {
+  if (A == nullptr || W == nullptr || bias == nullptr || out == nullptr || status_dev == nullptr)
+    return fail(EAS_ERR_INVALID_ARG, "a required pointer is null");
+  if (M <= 0 || N <= 0 || K <= 0 || K % 64 != 0 || N % 32 != 0) return fail(EAS_ERR_INVALID_ARG, "need M,N,K > 0, K %% 64 == 0, N %% 32 == 0");
+  if (act < 0 || act > 2 || (act == ACT_SWIGLU && out_fp32)) return fail(EAS_ERR_INVALID_ARG, "bad epilogue selection");
+  int budget = 0;
+  EAS_TRY(resolve_budget(sm_budget, &budget));
+  EAS_TRY(set_kernel_attributes());
+  Linear L;
+  L.w = static_cast<const bf16*>(W); L.b = static_cast<const bf16*>(bias); L.N = N; L.K = K;
+  EAS_TRY(finish_linear(L));
+  GemmCall g;
+  g.A = A; g.a_run = K; g.a_row_elems = K; g.a_rows = M; g.M = M; g.lin = &L; g.act = act; g.out_fp32 = out_fp32;
+  g.out = out; g.ldo = act == ACT_SWIGLU ? N / 2 : N; g.resid = out_fp32 ? resid : nullptr;
+  return launch_gemm(g, budget, static_cast<cudaStream_t>(stream), status_dev);
+}
+
+extern "C" eas_status eas_kernel_norm(const float* x, void* y, const void* gamma, const void* beta, int32_t rows, int32_t d,
+                                      int32_t kind, float eps, int32_t out_fp32, int32_t sm_budget, void* stream) {
+  if (x == nullptr || y == nullptr || rows <= 0) return fail(EAS_ERR_INVALID_ARG, "bad arguments");
+  if ((kind == NORM_LN && (gamma == nullptr || beta == nullptr)) || (kind == NORM_RMS && gamma == nullptr))
+    return fail(EAS_ERR_INVALID_ARG, "gamma/beta missing");
+  int budget = 0;
+  EAS_TRY(resolve_budget(sm_budget, &budget));
+  NormParams np{x, y, static_cast<const bf16*>(gamma), static_cast<const bf16*>(beta), nullptr, rows, d, eps};
+  return launch_norm(kind, out_fp32 != 0, np, budget, static_cast<cudaStream_t>(stream));
+}
+
+extern "C" eas_status eas_kernel_attention(const void* qkv, void* out, const int32_t* cu, int32_t n_items, int32_t n_heads,
+                                           int32_t head_dim, int32_t sm_budget, void* stream, int32_t impl, uint32_t* status_dev) {
+  if (qkv == nullptr || out == nullptr || cu == nullptr || status_dev == nullptr) return fail(EAS_ERR_INVALID_ARG, "a required pointer is null");
+  if (n_items < 1 || n_items > EAS_MAX_ITEMS || n_heads <= 0) return fail(EAS_ERR_INVALID_ARG, "bad sizes");
+  if (head_dim != 64 && head_dim != 80) return fail(EAS_ERR_UNSUPPORTED, "head_dim %d", head_dim);
+  for (int i = 0; i < n_items; ++i)
+    if (cu[i + 1] <= cu[i]) return fail(EAS_ERR_INVALID_ARG, "cu_seqlens is not strictly increasing");
+  int budget = 0;
+  EAS_TRY(resolve_budget(sm_budget, &budget));
+  return launch_attention(static_cast<const bf16*>(qkv), static_cast<bf16*>(out), cu, n_items, n_heads, head_dim, budget,
+                          static_cast<cudaStream_t>(stream), impl, status_dev);
+}

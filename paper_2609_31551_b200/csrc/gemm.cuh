@@ -1,0 +1,290 @@
+// Persistent bf16 GEMM for sm_100a:  D[M,N] = A[M,K] * W[N,K]^T  with a fused epilogue.
+//
+//   warp 0      TMA producer: 128x64 A tiles and 256x64 W tiles into a 4-stage shared-memory ring
+//   warp 1      UMMA issuer: tcgen05.mma 128x256x16, fp32 accumulators in TMEM, two accumulator
+//               buffers (2 x 256 columns) so that the epilogue of tile i overlaps the main loop of tile i+1
+//   warps 2..9  epilogue: tcgen05.ld -> bias / activation / rotary / residual -> global stores
+//
+// The grid is `sm_budget` CTAs (one per SM: the shared-memory request excludes a second resident
+// CTA) and each CTA walks tiles  blockIdx.x, blockIdx.x + gridDim.x, ...  in a fixed order, so the
+// result never depends on the budget: no split-K, no atomics.
+#pragma once
+#include "ptx.cuh"
+
+namespace eas {
+
+constexpr int kBM = 128, kBN = 256, kBK = 64;
+constexpr int kStages = 4;
+constexpr int kEpiWarps = 8;
+constexpr int kGemmThreads = 64 + 32 * kEpiWarps;
+constexpr int kABytes = kBM * kBK * 2;            // 16 KB
+constexpr int kBBytes = kBN * kBK * 2;            // 32 KB
+constexpr int kStageBytes = kABytes + kBBytes;    // 48 KB
+constexpr int kGemmSmemBytes = kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
+constexpr int kTmemCols = 512;
+constexpr int kPanelM = 8;                        // m-blocks per rasterisation panel (L2 reuse of W tiles)
+
+enum { ACT_NONE = 0, ACT_GELU = 1, ACT_SWIGLU = 2 };
+enum { OUT_BF16 = 0, OUT_F32 = 1 };
+
+struct alignas(64) GemmParams {
+  CUtensorMap tma_a;      // 3-D: {K-run, phase, rows}; box {64, 1, 128}
+  CUtensorMap tma_b;      // 2-D: {K, N}; box {64, 256}
+  int M, N;               // rows of A walked by tiles; rows of W
+  int k_blocks;           // K / 64 (K padded with zeros by the caller or by TMA fill)
+  int kb_per_tap;         // k-blocks per convolution tap (== k_blocks for a plain GEMM)
+  int conv_stride;        // 1 for a plain GEMM; row stride of a convolution otherwise
+  int m_blocks, n_blocks;
+  const bf16* bias;       // [N] (for SWIGLU: interleaved gate/up like the W rows)
+  void* out;              // bf16 or fp32 [*, ldo]
+  long long ldo;          // leading dimension of out (elements)
+  const float* resid;     // optional fp32 [*, ldo] added to the result (may alias out)
+  const int* row_map;     // optional: output row of each A row, negative = drop the row
+  const int* pos_idx;     // optional (with pos): row of the position table added to each A row
+  const bf16* pos;        // optional position table [*, N]
+  const float2* rope_cs;  // optional (cos, sin) per (A row, pair): columns < rope_ncols are rotated as adjacent pairs
+  int rope_pairs;         // pairs per head (head_dim / 2)
+  int rope_ncols;         // rotate output columns [0, rope_ncols)
+  int head_dim;
+  uint32_t* status;       // device status word
+};
+
+__device__ __forceinline__ void tile_coords(int tile, int m_blocks, int n_blocks, int& mb, int& nb) {
+  const int per_panel = kPanelM * n_blocks;
+  const int panel = tile / per_panel;
+  const int within = tile - panel * per_panel;
+  const int rows_here = min(kPanelM, m_blocks - panel * kPanelM);
+  nb = within / rows_here;
+  mb = panel * kPanelM + (within - nb * rows_here);
+}
+
+template <int ACT, int OUT>
+__global__ void __launch_bounds__(kGemmThreads, 1) gemm_kernel(const __grid_constant__ GemmParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  // 1024-byte alignment: the 128-byte swizzle pattern repeats every 8 rows of 128 bytes
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kStages * kStageBytes);
+  uint64_t* full_bar = bars;                    // [kStages]  TMA -> MMA
+  uint64_t* empty_bar = bars + kStages;         // [kStages]  MMA -> TMA
+  uint64_t* acc_full = bars + 2 * kStages;      // [2]        MMA -> epilogue
+  uint64_t* acc_empty = bars + 2 * kStages + 2; // [2]        epilogue -> MMA
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kStages + 4);
+  volatile uint32_t* abort_flag = tmem_slot + 1;
+
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+  const int num_tiles = p.m_blocks * p.n_blocks;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kStages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
+    for (int a = 0; a < 2; ++a) { mbar_init(&acc_full[a], 1); mbar_init(&acc_empty[a], kEpiWarps); }
+    *abort_flag = 0;
+    mbar_fence_init();
+    tma_prefetch_desc(&p.tma_a);
+    tma_prefetch_desc(&p.tma_b);
+  }
+  if (warp == 1) {
+    tmem_alloc(tmem_slot, kTmemCols);
+    tmem_relinquish();
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ producer
+    if (lane == 0) {
+      uint32_t it = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+        int mb, nb;
+        tile_coords(tile, p.m_blocks, p.n_blocks, mb, nb);
+        for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
+          const int s = it % kStages;
+          const uint32_t ph = (it / kStages) & 1u;
+          if (!mbar_wait(&empty_bar[s], ph ^ 1u, abort_flag)) { ok = false; break; }
+          uint8_t* sa = smem + s * kStageBytes;
+          uint8_t* sb = sa + kABytes;
+          mbar_expect_tx(&full_bar[s], kStageBytes);
+          const int tap = kb / p.kb_per_tap;
+          const int kx = (kb - tap * p.kb_per_tap) * kBK;
+          tma_load_3d(sa, &p.tma_a, &full_bar[s], kx, tap % p.conv_stride, mb * kBM + tap / p.conv_stride);
+          tma_load_2d(sb, &p.tma_b, &full_bar[s], kb * kBK, nb * kBN);
+        }
+      }
+      if (!ok) {
+        // give loads already in flight a bounded chance to land before the CTA retires
+        for (int s = 0; s < kStages; ++s) {
+          const long long t0 = clock64();
+          while (clock64() - t0 < 2000000) {}
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ UMMA issuer
+    if (lane == 0) {
+      constexpr uint32_t idesc = make_idesc_bf16(kBM, kBN, 0, 0);
+      uint32_t it = 0, tcount = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++tcount) {
+        const uint32_t acc = tcount & 1u;
+        const uint32_t acc_ph = (tcount >> 1) & 1u;
+        if (!mbar_wait(&acc_empty[acc], acc_ph ^ 1u, abort_flag)) { ok = false; break; }
+        tc_fence_after_sync();
+        const uint32_t tmem_d = tmem_base + acc * kBN;
+        for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
+          const int s = it % kStages;
+          const uint32_t ph = (it / kStages) & 1u;
+          if (!mbar_wait(&full_bar[s], ph, abort_flag)) { ok = false; break; }
+          tc_fence_after_sync();
+          const uint32_t a_addr = smem_u32(smem + s * kStageBytes);
+          const uint32_t b_addr = a_addr + kABytes;
+          const uint64_t adesc = make_smem_desc(a_addr, 16, 1024, kSwizzle128B);
+          const uint64_t bdesc = make_smem_desc(b_addr, 16, 1024, kSwizzle128B);
+#pragma unroll
+          for (int k = 0; k < kBK / 16; ++k) {
+            // advancing 16 bf16 = 32 bytes along K inside the swizzle atom: +2 in the (>>4) address field
+            umma_bf16_ss(tmem_d, adesc + 2 * k, bdesc + 2 * k, idesc, (kb | k) != 0);
+          }
+          umma_commit(&empty_bar[s]);           // frees the stage once these UMMAs have read it
+        }
+        if (ok) umma_commit(&acc_full[acc]);    // accumulator complete
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ epilogue
+    const int ew = warp - 2;                    // 0..7
+    const int quarter = warp & 3;               // TMEM lane quarter this warp may read
+    const int half = ew >> 2;                   // which 128 accumulator columns
+    uint32_t tcount = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++tcount) {
+      int mb, nb;
+      tile_coords(tile, p.m_blocks, p.n_blocks, mb, nb);
+      const uint32_t acc = tcount & 1u;
+      const uint32_t acc_ph = (tcount >> 1) & 1u;
+      if (!mbar_wait(&acc_full[acc], acc_ph, abort_flag)) { ok = false; break; }
+      tc_fence_after_sync();
+
+      const int arow = mb * kBM + quarter * 32 + lane;            // row of A (== accumulator row)
+      long long orow = arow;
+      bool row_ok = arow < p.M;
+      if (row_ok && p.row_map != nullptr) {
+        const int mapped = p.row_map[arow];
+        row_ok = mapped >= 0;
+        orow = mapped;
+      }
+      const int posrow = (row_ok && p.pos_idx != nullptr) ? p.pos_idx[arow] : 0;
+
+#pragma unroll 1
+      for (int c = 0; c < 4; ++c) {
+        const int col_in_tile = half * 128 + c * 32;
+        const int col0 = nb * kBN + col_in_tile;                  // first of 32 output-space accumulator columns
+        uint32_t raw[32];
+        __syncwarp();   // the TMEM load is warp-collective: reconverge after the per-row branches below
+        tmem_ld_32x32(tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + acc * kBN + col_in_tile, raw);
+        tmem_ld_wait();
+        if (!row_ok || col0 >= p.N) continue;
+        float v[32];
+#pragma unroll
+        for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(raw[i]);
+        {  // bias: 32 bf16 = 64 bytes, the same for every row
+          const uint4* bp = reinterpret_cast<const uint4*>(p.bias + col0);
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            const uint4 b = __ldg(bp + q);
+            const uint32_t w[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              v[q * 8 + 2 * j] += bf16_lo(w[j]);
+              v[q * 8 + 2 * j + 1] += bf16_hi(w[j]);
+            }
+          }
+        }
+        if (p.rope_cs != nullptr && col0 < p.rope_ncols) {
+          // rotary: adjacent columns (2i, 2i+1) of a head form pair i (the weight rows were
+          // re-ordered at create time so that the two halves of a pair sit side by side)
+          const float2* cs = p.rope_cs + static_cast<long long>(arow) * p.rope_pairs;
+          int pi = (col0 % p.head_dim) >> 1;
+#pragma unroll
+          for (int j = 0; j < 16; ++j) {
+            const float2 t = __ldg(cs + pi);
+            const float x0 = v[2 * j], x1 = v[2 * j + 1];
+            v[2 * j] = x0 * t.x - x1 * t.y;
+            v[2 * j + 1] = x1 * t.x + x0 * t.y;
+            if (++pi == p.rope_pairs) pi = 0;
+          }
+        }
+        if (ACT == ACT_GELU) {
+#pragma unroll
+          for (int i = 0; i < 32; ++i) v[i] = gelu_erf(v[i]);
+        }
+        if (ACT == ACT_SWIGLU) {
+          // columns (2j, 2j+1) = (gate_j, up_j); 16 outputs per 32 accumulator columns
+          bf16* o = reinterpret_cast<bf16*>(p.out) + orow * p.ldo + (col0 >> 1);
+          uint32_t w[8];
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            const float a0 = silu_f(v[4 * j]) * v[4 * j + 1];
+            const float a1 = silu_f(v[4 * j + 2]) * v[4 * j + 3];
+            w[j] = pack_bf16x2(a0, a1);
+          }
+          uint4* o4 = reinterpret_cast<uint4*>(o);
+          o4[0] = make_uint4(w[0], w[1], w[2], w[3]);
+          o4[1] = make_uint4(w[4], w[5], w[6], w[7]);
+          continue;
+        }
+        if (p.pos != nullptr) {
+          const uint4* pp = reinterpret_cast<const uint4*>(p.pos + static_cast<long long>(posrow) * p.N + col0);
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            const uint4 b = __ldg(pp + q);
+            const uint32_t w[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              v[q * 8 + 2 * j] += bf16_lo(w[j]);
+              v[q * 8 + 2 * j + 1] += bf16_hi(w[j]);
+            }
+          }
+        }
+        if (OUT == OUT_F32) {
+          float* o = reinterpret_cast<float*>(p.out) + orow * p.ldo + col0;
+          if (p.resid != nullptr) {
+            const float4* r4 = reinterpret_cast<const float4*>(p.resid + orow * p.ldo + col0);
+#pragma unroll
+            for (int q = 0; q < 8; ++q) {
+              const float4 r = r4[q];
+              v[4 * q] += r.x; v[4 * q + 1] += r.y; v[4 * q + 2] += r.z; v[4 * q + 3] += r.w;
+            }
+          }
+          float4* o4 = reinterpret_cast<float4*>(o);
+#pragma unroll
+          for (int q = 0; q < 8; ++q) o4[q] = make_float4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
+        } else {
+          bf16* o = reinterpret_cast<bf16*>(p.out) + orow * p.ldo + col0;
+          uint4* o4 = reinterpret_cast<uint4*>(o);
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            o4[q] = make_uint4(pack_bf16x2(v[8 * q], v[8 * q + 1]), pack_bf16x2(v[8 * q + 2], v[8 * q + 3]),
+                               pack_bf16x2(v[8 * q + 4], v[8 * q + 5]), pack_bf16x2(v[8 * q + 6], v[8 * q + 7]));
+          }
+        }
+      }
+      // all TMEM reads of this warp are complete (wait::ld above): hand the accumulator back
+      tc_fence_before_sync();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&acc_empty[acc]);
+    }
+  }
+
+  tc_fence_before_sync();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after_sync();
+    tmem_dealloc(tmem_base, kTmemCols);
+  }
+  if (threadIdx.x == 0 && *abort_flag) atomicCAS(p.status, DEV_OK, DEV_ERR_WAIT_TIMEOUT);
+}
+
+}  // namespace eas

@@ -1,0 +1,82 @@
+"""Whole-encoder parity: the CUDA path through the C ABI against the fp64 oracle, element by element
+on the same seeded inputs, for all five workload families; plus the determinism properties."""
+import numpy as np
+import pytest
+import torch
+
+import eas_synth as S
+from oracle import encoder_oracle as O
+from tests import gpu_util as G
+
+pytestmark = pytest.mark.gpu
+
+
+def _make(cfg, profile="plain"):
+    import paper_2609_31551_b200 as P
+    w = S.make_weights(cfg, profile=profile)
+    enc = P.Encoder(cfg, P.weights_to_device(w))
+    return w, enc
+
+
+CASES = {
+    # name: (config overrides, item shapes)
+    "c0_full": ("c0", {}, [(1, 224, 224)] * 4),
+    "c1_2layers": ("c1", dict(n_layers=2), [(1, 336, 336)] * 3),
+    "c2_2layers": ("c2", dict(n_layers=2), [(1, 56, 84), (1, 224, 224), (1, 28, 28), (1, 140, 364)]),
+    "c3_2layers": ("c3", dict(n_layers=2), [(4, 56, 56), (2, 112, 84)]),
+    "c4_2layers": ("c4", dict(n_layers=2, max_pos=1500), [(200, 128, 1), (600, 128, 1), (2, 128, 1)]),
+}
+
+
+@pytest.mark.parametrize("case", list(CASES))
+@pytest.mark.parametrize("profile", ["plain", "sharp"])
+def test_encoder_parity_small(case, profile):
+    name, over, shapes = CASES[case]
+    cfg = S.get_config(name, **over)
+    w, enc = _make(cfg, profile)
+    items = S.make_items(cfg, shapes, seed=2000 + len(shapes))
+    ref, cu, _ = O.encode_microbatch(cfg, w, items)
+    got, _ = G.run_gpu(enc, cfg, items)
+    rel, mabs = G.assert_parity(got, ref, case)
+    print(f"{case}/{profile}: row-rel {rel:.3e} max-abs {mabs:.3e}")
+
+
+def test_c0_bit_stability_and_packing_invariance():
+    cfg = S.get_config("c0")
+    w, enc = _make(cfg)
+    items = S.make_items(cfg, [(1, 224, 224)] * 4, seed=2002)
+    _, a = G.run_gpu(enc, cfg, items)
+    _, b = G.run_gpu(enc, cfg, items)
+    assert torch.equal(a, b)                                  # same input twice -> same bytes
+    for budget in (37, 74, 111):
+        _, c = G.run_gpu(enc, cfg, items, sm_budget=budget)
+        assert torch.equal(a, c), budget                      # any sm_budget -> same bytes
+    _, alone = G.run_gpu(enc, cfg, [items[2]])
+    assert torch.equal(a[2 * 196:3 * 196], alone)             # item alone == item packed
+
+
+def test_invalid_arguments_are_rejected_before_launch():
+    import paper_2609_31551_b200 as P
+    cfg = S.get_config("c0")
+    w, enc = _make(cfg)
+    items = S.make_items(cfg, [(1, 224, 224)], seed=1)
+    data, offs = P.pack_items(items)
+    with pytest.raises(P.EasError) as e:
+        enc.encode_microbatch(data, [(1, 224, 224)], offs, [0, 195])
+    assert e.value.status == 1
+    with pytest.raises(P.EasError) as e:
+        enc.encode_microbatch(data, [(1, 224, 230)], offs, [0, 196])
+    assert e.value.status == 1
+    with pytest.raises(P.EasError) as e:
+        enc.encode_microbatch(data, [(1, 224, 224)], offs, [0, 196], sm_budget=100000)
+    assert e.value.status == 1
+    small = torch.empty(1024, dtype=torch.uint8, device="cuda")
+    with pytest.raises(P.EasError) as e:
+        enc.encode_microbatch(data, [(1, 224, 224)], offs, [0, 196], workspace=small)
+    assert e.value.status == 3
+    # a device cu_seqlens that differs from the host copy is reported by the device check
+    bad = torch.tensor([0, 100], dtype=torch.int32, device="cuda")
+    enc.encode_microbatch(data, [(1, 224, 224)], offs, [0, 196], cu_seqlens_dev=bad)
+    with pytest.raises(P.EasError) as e:
+        enc.status()
+    assert e.value.status == 7

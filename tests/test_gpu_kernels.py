@@ -1,0 +1,106 @@
+"""Single-kernel parity: each CUDA kernel, called through the C ABI, against the oracle's definition
+of the same operation on seeded inputs.  Shapes span several tiles, ragged tails and tiny cases."""
+import numpy as np
+import pytest
+import torch
+
+import eas_synth as S
+from oracle import encoder_oracle as O
+
+pytestmark = pytest.mark.gpu
+
+
+def _bf16_exact(rng, shape, scale=1.0):
+    return S.round_to_bf16((rng.standard_normal(shape) * scale).astype(np.float32))
+
+
+def _dev(a):
+    return torch.from_numpy(a).to("cuda", dtype=torch.bfloat16)
+
+
+@pytest.mark.parametrize("M,N,K", [(784, 256, 768), (300, 512, 128), (129, 256, 64), (1, 32, 64), (257, 96, 640),
+                                   (1000, 1024, 1024), (128, 3072, 256), (77, 288, 192)])
+@pytest.mark.parametrize("act,out_fp32", [(0, False), (1, False), (2, False), (0, True)])
+def test_gemm_epilogues(M, N, K, act, out_fp32):
+    import paper_2609_31551_b200 as P
+    rng = np.random.Generator(np.random.PCG64(M * 7 + N * 3 + K + act))
+    A, W, b = _bf16_exact(rng, (M, K)), _bf16_exact(rng, (N, K), 0.05), _bf16_exact(rng, (N,), 0.5)
+    y = O.linear(O._t(A), O._t(W), O._t(b))
+    resid = None
+    if act == 1:
+        y = O.gelu(y)
+    if act == 2:
+        y = O.silu(y[:, 0::2]) * y[:, 1::2]          # interleaved (gate_j, up_j) rows
+    if out_fp32:
+        r = rng.standard_normal((M, N)).astype(np.float32)
+        resid = torch.from_numpy(r).cuda()
+        y = y + O._t(r)
+    out, status = P.kernel_gemm(_dev(A), _dev(W), _dev(b), act=act, out_fp32=out_fp32, resid=resid)
+    torch.cuda.synchronize()
+    assert int(status[0]) == 0
+    got = out.double().cpu()
+    # fp32 accumulation over K, then one rounding (bf16: 2^-9 relative; fp32 output: accumulation only)
+    tol = (1e-5 if out_fp32 else 2.0 ** -8) * y.abs() + 2e-3 * max(1.0, float(K) ** 0.5 * 0.05)
+    bad = (got - y).abs() > tol
+    assert not bad.any(), f"{int(bad.sum())} of {bad.numel()} wrong, max err {(got - y).abs().max():.4e}, first bad {bad.nonzero()[:5].tolist()}"
+
+
+def test_gemm_is_independent_of_sm_budget():
+    import paper_2609_31551_b200 as P
+    rng = np.random.Generator(np.random.PCG64(5))
+    A, W, b = _dev(_bf16_exact(rng, (1500, 512))), _dev(_bf16_exact(rng, (768, 512), 0.05)), _dev(_bf16_exact(rng, (768,)))
+    ref, _ = P.kernel_gemm(A, W, b, act=1)
+    for budget in (1, 7, 37, 74, 111):
+        out, _ = P.kernel_gemm(A, W, b, act=1, sm_budget=budget)
+        assert torch.equal(out, ref), budget
+
+
+@pytest.mark.parametrize("d", [256, 1024, 1280])
+@pytest.mark.parametrize("kind", [0, 1, 2])
+def test_norm(d, kind):
+    import paper_2609_31551_b200 as P
+    rng = np.random.Generator(np.random.PCG64(d + kind))
+    rows = 1003
+    x = (rng.standard_normal((rows, d)) * 3 + 0.7).astype(np.float32)
+    g, b = _bf16_exact(rng, (d,), 0.1) + 1, _bf16_exact(rng, (d,), 0.1)
+    g = S.round_to_bf16(g)
+    eps = 1e-5 if kind == 0 else 1e-6
+    if kind == 0:
+        ref = O.layer_norm(O._t(x), O._t(g), O._t(b), eps)
+    elif kind == 1:
+        ref = O.rms_norm(O._t(x), O._t(g), eps)
+    else:
+        ref = O._t(x)
+    xd = torch.from_numpy(x).cuda()
+    y = P.kernel_norm(xd, _dev(g), _dev(b), kind, eps)
+    y32 = P.kernel_norm(xd, _dev(g), _dev(b), kind, eps, out_fp32=True) if kind != 2 else None
+    torch.cuda.synchronize()
+    assert (y.double().cpu() - ref).abs().max() <= 2.0 ** -8 * ref.abs().max() + 1e-6
+    if y32 is not None:
+        assert (y32.double().cpu() - ref).abs().max() <= 2e-5 * max(1.0, float(ref.abs().max()))
+    y2 = P.kernel_norm(xd, _dev(g), _dev(b), kind, eps, sm_budget=5)
+    assert torch.equal(y, y2)
+
+
+@pytest.mark.parametrize("hd,H", [(64, 3), (80, 2)])
+@pytest.mark.parametrize("lens", [[5], [128], [129, 1, 64, 577], [200, 1000]])
+@pytest.mark.parametrize("impl", [0, 1])
+def test_attention_block_diagonal(hd, H, lens, impl):
+    import paper_2609_31551_b200 as P
+    rng = np.random.Generator(np.random.PCG64(hd + len(lens) + sum(lens)))
+    T, d = sum(lens), H * hd
+    qkv = _bf16_exact(rng, (T, 3 * d))
+    qkv[:, : 2 * d] *= 1.5            # sharp softmax: score std about 2
+    qkv = S.round_to_bf16(qkv)
+    cu = np.concatenate([[0], np.cumsum(lens)]).astype(np.int32)
+    q = O._t(qkv)
+    ref = torch.cat([O.attention_one_item(q[a:b, :d].reshape(-1, H, hd), q[a:b, d:2 * d].reshape(-1, H, hd),
+                                          q[a:b, 2 * d:].reshape(-1, H, hd)) for a, b in zip(cu[:-1], cu[1:])])
+    out, status = P.kernel_attention(_dev(qkv), cu, H, hd, impl=impl)
+    torch.cuda.synchronize()
+    assert int(status[0]) == 0
+    err = (out.double().cpu() - ref).abs().max()
+    # P is rounded to bf16 before P*V and the output to bf16: a few 2^-9 of |v| <= ~4
+    assert err <= 2e-2, err
+    out2, _ = P.kernel_attention(_dev(qkv), cu, H, hd, impl=impl, sm_budget=3)
+    assert torch.equal(out, out2)
