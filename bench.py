@@ -1,0 +1,373 @@
+#!/usr/bin/env python
+"""Benchmark of the Encode-stage forward pass (one step = one micro-batch through the whole encoder).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config c1] [--micro-batch 32] [--sm-budget 0]
+    python bench.py --impl reference ...      # times the CPU fp64 oracle on a bounded sample
+
+Prints ONE JSON line.  `value` is encoder tokens/s with inputs resident in HBM; `e2e` is the same metric
+through the C ABI with host buffers (pinned host -> device copy of the pixels and device -> host copy of the
+embeddings inside the timed region, double-buffered on copy streams); `roofline` is the dominant kernel class
+(the GEMMs) timed with CUDA events inside the library; `cpu_baseline` is the oracle on this machine's host cores.
+Multi-GPU: replicas only (items are independent, the path has no collective); each rank encodes its own
+micro-batches and the job value is the sum of tokens over the slowest rank's time."""
+from __future__ import annotations
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import eas_synth as S  # noqa: E402
+
+
+# ------------------------------------------------------------------ algorithmic work (real tokens only)
+def flops_of(cfg, shapes):
+    """Algorithmic FLOPs of one forward pass: 2*M*N*K per linear map, 4*d*S^2 per item and layer for attention."""
+    d, I, L = cfg["d_model"], cfg["d_mlp"], cfg["n_layers"]
+    seqs = [S.tokens_per_item(cfg, s) for s in shapes]
+    T = sum(seqs)
+    mlp = (6 if cfg["mlp"] == 1 else 4) * d * I
+    lin = L * T * (8 * d * d + mlp)
+    attn = L * 4 * d * sum(s * s for s in seqs)
+    if cfg["family"] == 2:
+        emb = sum(2 * s[0] * 3 * cfg["in_channels"] * d + 2 * (s[0] // 2) * 3 * d * d for s in shapes)
+    else:
+        emb = 2 * (T - (len(shapes) if cfg["has_cls"] else 0)) * S.configs.embed_k(cfg) * d
+    head = 0
+    out_rows = sum(S.out_tokens_per_item(cfg, s) for s in shapes)
+    if cfg["head"] == 1:
+        head = 2 * out_rows * (d * cfg["d_head_hidden"] + cfg["d_head_hidden"] * cfg["d_out"])
+    elif cfg["head"] == 2:
+        head = 2 * out_rows * (4 * d * cfg["d_head_hidden"] + cfg["d_head_hidden"] * cfg["d_out"])
+    return dict(total=lin + attn + emb + head, linear=lin + emb + head, attention=attn, tokens=T, out_rows=out_rows,
+                sum_s2=sum(s * s for s in seqs))
+
+
+def gemm_flops_by_class(cfg, shapes):
+    """Algorithmic FLOPs per kernel class of the GEMMs (keys = EAS_KC_* ids)."""
+    d, I, L = cfg["d_model"], cfg["d_mlp"], cfg["n_layers"]
+    f = flops_of(cfg, shapes)
+    T = f["tokens"]
+    up = (4 if cfg["mlp"] == 1 else 2) * d * I
+    emb = f["linear"] - L * T * (8 * d * d + (6 if cfg["mlp"] == 1 else 4) * d * I)
+    head = 0
+    if cfg["head"]:
+        kin = 4 * d if cfg["head"] == 2 else d
+        head = 2 * f["out_rows"] * (kin * cfg["d_head_hidden"] + cfg["d_head_hidden"] * cfg["d_out"])
+    return {2: emb - head, 4: L * T * 6 * d * d, 6: L * T * 2 * d * d, 7: L * T * up, 8: L * T * 2 * d * I, 9: head,
+            5: f["attention"]}
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.gpu}", f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons, pw = [], [], set(), []
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            parts = [p.strip() for p in ln.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0])); mx.append(float(parts[1])); pw.append(float(parts[2]))
+            except ValueError:
+                continue
+            for nm, val in zip(names, parts[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(nm)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "power_w_max": max(pw) if pw else None, "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return dict(hbm=p["hbm_gbs"], burst=p["bf16_tflops"], sustained=p["bf16_tflops_sustained"], source="measured")
+    return dict(hbm=6650.0, burst=1590.0, sustained=1400.0, source="fallback")
+
+
+def workload(cfg_name, mb, seed_shift=0):
+    cfg = S.get_config(cfg_name)
+    ci = S.configs.CONFIG_INDEX[cfg_name]
+    lg = int(np.log2(max(mb, 1)))
+    shapes = S.draw_item_shapes(cfg, mb, 3000 + 100 * ci + lg + seed_shift)
+    return cfg, shapes, 2000 + 100 * ci + lg + seed_shift
+
+
+# ------------------------------------------------------------------ reference arm: the oracle on host cores
+def run_reference(args):
+    import torch
+    from oracle import encoder_oracle as O
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    cfg, shapes, seed = workload(args.config, args.micro_batch)
+    sample_shapes = shapes[:1]          # bounded sample: the first item of the micro-batch
+    w = S.make_weights(cfg)
+    items = S.make_items(cfg, sample_shapes, seed)
+    f = flops_of(cfg, sample_shapes)
+    for _ in range(args.warmup):
+        O.encode_microbatch(cfg, w, items)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        O.encode_microbatch(cfg, w, items)
+    dt = (time.perf_counter() - t0) / args.steps
+    val = f["tokens"] / dt
+    line = {"impl": "reference", "metric": "encoder_tokens_per_sec", "value": val, "unit": "tokens/s", "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": f"{args.config} micro-batch {args.micro_batch} (sample: 1 item per step)"},
+            "cpu_baseline": {"value": val, "unit": "tokens/s", "cores": torch.get_num_threads(), "kind": "oracle",
+                             "sample": f"1 item ({f['tokens']} tokens) of the {args.config} micro-batch per step"},
+            "e2e": {"value": val, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+# ------------------------------------------------------------------ CUDA arm
+def run_cuda(args):
+    import torch
+    import torch.distributed as dist
+    import paper_2609_31551_b200 as P
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: the encoder has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+
+    cfg, shapes, seed = workload(args.config, args.micro_batch, seed_shift=1000 * rank)
+    w = S.make_weights(cfg)
+    enc = P.Encoder(cfg, P.weights_to_device(w))
+    items = S.make_items(cfg, shapes, seed)
+    data, offsets = P.pack_items(items)
+    cu = np.concatenate([[0], np.cumsum([S.tokens_per_item(cfg, s) for s in shapes])]).astype(np.int32)
+    cu_dev = torch.from_numpy(cu).cuda()
+    f = flops_of(cfg, shapes)
+    T = f["tokens"]
+    budget = args.sm_budget
+    stream = torch.cuda.current_stream()
+    out = torch.empty((f["out_rows"], cfg["d_out"]), dtype=torch.bfloat16, device="cuda")
+
+    def step():
+        enc.encode_microbatch(data, shapes, offsets, cu, cu_seqlens_dev=cu_dev, sm_budget=budget, out=out)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    enc.status()
+
+    # ---- value: inputs resident in HBM
+    sampler = ClockSampler(local_rank)
+    barrier()
+    sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(args.steps):
+        step()
+    e1.record(stream)
+    barrier()
+    ms = e0.elapsed_time(e1)
+    enc.status()
+    launches = enc.last_launch_count() * args.steps
+
+    # ---- e2e: host buffers, copies inside the timed region, double-buffered
+    host_in = torch.empty(data.numel(), dtype=torch.bfloat16, pin_memory=True)
+    host_in.copy_(data.cpu())
+    host_out = [torch.empty(out.shape, dtype=torch.bfloat16, pin_memory=True) for _ in range(2)]
+    dev_in = [torch.empty_like(data) for _ in range(2)]
+    dev_out = [torch.empty_like(out) for _ in range(2)]
+    s_in, s_out = torch.cuda.Stream(), torch.cuda.Stream()
+    ev_in = [torch.cuda.Event() for _ in range(2)]
+    ev_done = [torch.cuda.Event() for _ in range(2)]
+    ev_free_in = [torch.cuda.Event() for _ in range(2)]
+    ev_free_out = [torch.cuda.Event() for _ in range(2)]
+
+    def e2e_loop(n):
+        for i in range(n):
+            b = i & 1
+            with torch.cuda.stream(s_in):
+                if i >= 2:
+                    s_in.wait_event(ev_free_in[b])
+                dev_in[b].copy_(host_in, non_blocking=True)
+                ev_in[b].record(s_in)
+            stream.wait_event(ev_in[b])
+            if i >= 2:
+                stream.wait_event(ev_free_out[b])
+            enc.encode_microbatch(dev_in[b], shapes, offsets, cu, cu_seqlens_dev=cu_dev, sm_budget=budget, out=dev_out[b])
+            ev_done[b].record(stream)
+            ev_free_in[b].record(stream)
+            with torch.cuda.stream(s_out):
+                s_out.wait_event(ev_done[b])
+                host_out[b].copy_(dev_out[b], non_blocking=True)
+                ev_free_out[b].record(s_out)
+
+    e2e_loop(2)
+    barrier()
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0.record(stream)
+    e2e_loop(args.steps)
+    s_out.wait_stream(stream)
+    t1.record(s_out)
+    barrier()
+    ms_e2e = t0.elapsed_time(t1)
+    clocks = sampler.stop()
+    h2d = data.numel() * 2
+    d2h = out.numel() * 2
+
+    # ---- per-kernel-class timing (separate pass over the same workload, events inside the library)
+    enc.enable_timing(True)
+    acc = {}
+    n_prof = min(args.steps, 5)
+    for _ in range(n_prof):
+        step()
+        cls, kms = enc.timing_read()
+        for c_, m_ in zip(cls.tolist(), kms.tolist()):
+            a = acc.setdefault(c_, [0.0, 0])
+            a[0] += m_; a[1] += 1
+    enc.enable_timing(False)
+    torch.cuda.synchronize()
+
+    if world > 1:
+        t = torch.tensor([ms, ms_e2e], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms, ms_e2e = t.tolist()
+        tok = torch.tensor([float(T)], dtype=torch.float64, device="cuda")
+        dist.all_reduce(tok)
+        total_tokens = tok.item()
+        nl = torch.tensor([float(launches)], dtype=torch.float64, device="cuda")
+        dist.all_reduce(nl)
+        launches = int(nl.item())
+    else:
+        total_tokens = float(T)
+
+    if rank == 0:
+        peaks = measured_peaks()
+        gf = gemm_flops_by_class(cfg, shapes)
+        gemm_ids = [2, 4, 6, 7, 8, 9]
+        gemm_ms = sum(acc[c_][0] for c_ in gemm_ids if c_ in acc) / n_prof
+        gemm_launch = sum(acc[c_][1] for c_ in gemm_ids if c_ in acc) / n_prof
+        gemm_fl = sum(gf[c_] for c_ in gemm_ids)
+        achieved = gemm_fl / (gemm_ms * 1e-3) / 1e12 if gemm_ms > 0 else 0.0
+        names = {0: "prep", 1: "embed_gather", 2: "gemm_embed", 3: "norm", 4: "gemm_qkv", 5: "attention", 6: "gemm_proj",
+                 7: "gemm_fc1", 8: "gemm_fc2", 9: "gemm_head"}
+        breakdown = {}
+        for c_, (tm, cnt) in sorted(acc.items()):
+            ent = {"ms_per_step": round(tm / n_prof, 4), "launches_per_step": cnt // n_prof}
+            if c_ in gf and tm > 0:
+                ent["tflops"] = round(gf[c_] / (tm / n_prof * 1e-3) / 1e12, 1)
+            breakdown[names.get(c_, str(c_))] = ent
+        step_ms = ms / args.steps
+        line = {
+            "metric": "encoder_tokens_per_sec", "value": total_tokens * args.steps / (ms * 1e-3), "unit": "tokens/s",
+            "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": step_ms,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": f"{args.config} micro-batch {args.micro_batch}", "items_per_step": len(shapes),
+                       "tokens_per_step": T, "sm_budget": budget if budget else "all",
+                       "l2": "working set (weights + activations) larger than L2; no flush",
+                       "parallelism": "replicas" if world > 1 else "single"},
+            "items_per_sec": len(shapes) * world * args.steps / (ms * 1e-3),
+            "tflops": f["total"] * world / (step_ms * 1e-3) / 1e12,
+            "frac_of_bf16_peak": {"burst_measured": f["total"] / (step_ms * 1e-3) / 1e12 / peaks["burst"],
+                                  "sustained_measured": f["total"] / (step_ms * 1e-3) / 1e12 / peaks["sustained"],
+                                  "source": peaks["source"]},
+            "e2e": {"value": total_tokens * args.steps / (ms_e2e * 1e-3), "unit": "tokens/s", "h2d_bytes_per_step": h2d,
+                    "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e / args.steps},
+            "gpu_launches": launches,
+            "clocks": clocks,
+            "roofline": {"bound": "tensor", "kernel": "gemm_kernel (all GEMM launches of a step)", "achieved": achieved,
+                         "peak": peaks["sustained"], "unit": "TFLOP/s", "frac": achieved / peaks["sustained"],
+                         "peak_kind": f"sustained bf16, {peaks['source']}", "traffic": None,
+                         "launches_per_step": gemm_launch, "avg_launch_ms": gemm_ms / max(gemm_launch, 1)},
+            "kernel_breakdown": breakdown,
+        }
+        if world == 1 and not args.no_cpu_baseline:
+            line["cpu_baseline"] = cpu_baseline(cfg, w, shapes, seed)
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def cpu_baseline(cfg, w, shapes, seed):
+    """The oracle, as it stands, on one item of the workload (a bounded sample of the same step)."""
+    import torch
+    from oracle import encoder_oracle as O
+    items = S.make_items(cfg, shapes[:1], seed)
+    f1 = flops_of(cfg, shapes[:1])
+    t0 = time.perf_counter()
+    n = 0
+    while True:
+        O.encode_microbatch(cfg, w, items)
+        n += 1
+        if time.perf_counter() - t0 > 10.0 or n >= 8:
+            break
+    dt = (time.perf_counter() - t0) / n
+    return {"value": f1["tokens"] / dt, "unit": "tokens/s", "cores": torch.get_num_threads(), "kind": "oracle",
+            "sample": f"{n} x 1 item ({f1['tokens']} tokens, {f1['total'] / 1e9:.0f} GFLOP fp64) of the step's micro-batch",
+            "gflops": f1["total"] / dt / 1e9}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
+    ap.add_argument("--config", default="c1", choices=["c0", "c1", "c2", "c3", "c4"])
+    ap.add_argument("--micro-batch", type=int, default=32)
+    ap.add_argument("--sm-budget", type=int, default=0)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_cuda(args)
+
+
+if __name__ == "__main__":
+    main()

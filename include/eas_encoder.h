@@ -145,6 +145,17 @@ int32_t eas_encoder_last_launch_count(const eas_encoder* enc);
 /* Selects the attention kernel: 0 = default; 1 = register-tile (mma.sync) kernel.  For testing. */
 eas_status eas_encoder_set_attention_impl(eas_encoder* enc, int32_t impl);
 
+/* Per-kernel timing for profiling (off by default; adds one event record per launch).  Kernel classes: */
+enum { EAS_KC_PREP = 0, EAS_KC_EMBED_GATHER = 1, EAS_KC_GEMM_EMBED = 2, EAS_KC_NORM = 3, EAS_KC_GEMM_QKV = 4,
+       EAS_KC_ATTENTION = 5, EAS_KC_GEMM_PROJ = 6, EAS_KC_GEMM_FC1 = 7, EAS_KC_GEMM_FC2 = 8, EAS_KC_GEMM_HEAD = 9,
+       EAS_KC_COUNT = 10 };
+/* on != 0: the following eas_encode_microbatch calls record a CUDA event in front of every launch. */
+eas_status eas_encoder_enable_timing(eas_encoder* enc, int32_t on);
+/* Waits for the last timed call, then writes the class and device milliseconds of its launches, in launch
+ * order, into host arrays of `capacity` entries.  Returns the number written (with NULL arrays: the number
+ * available), or -1 on a CUDA error. */
+int32_t eas_encoder_timing_read(eas_encoder* enc, int32_t capacity, int32_t* kernel_class, float* ms);
+
 const char* eas_last_error(void);
 
 void eas_encoder_destroy(eas_encoder* enc);

@@ -16,7 +16,7 @@ STATUS_NAMES = {0: "EAS_OK", 1: "EAS_ERR_INVALID_ARG", 2: "EAS_ERR_UNSUPPORTED",
 EXPORTED_SYMBOLS = [
     "eas_encoder_create", "eas_encoder_weight_arena_bytes", "eas_encoder_workspace_bytes", "eas_encoder_out_rows",
     "eas_encode_microbatch", "eas_encoder_status", "eas_encoder_last_launch_count", "eas_encoder_set_attention_impl",
-    "eas_last_error", "eas_encoder_destroy", "eas_kernel_gemm", "eas_kernel_norm", "eas_kernel_attention",
+    "eas_encoder_enable_timing", "eas_encoder_timing_read", "eas_last_error", "eas_encoder_destroy", "eas_kernel_gemm", "eas_kernel_norm", "eas_kernel_attention",
 ]
 
 
@@ -75,6 +75,10 @@ def load_library():
     lib.eas_encoder_last_launch_count.argtypes = [C.c_void_p]
     lib.eas_encoder_set_attention_impl.restype = C.c_int
     lib.eas_encoder_set_attention_impl.argtypes = [C.c_void_p, C.c_int32]
+    lib.eas_encoder_enable_timing.restype = C.c_int
+    lib.eas_encoder_enable_timing.argtypes = [C.c_void_p, C.c_int32]
+    lib.eas_encoder_timing_read.restype = C.c_int32
+    lib.eas_encoder_timing_read.argtypes = [C.c_void_p, C.c_int32, C.POINTER(C.c_int32), C.POINTER(C.c_float)]
     lib.eas_last_error.restype = C.c_char_p
     lib.eas_last_error.argtypes = []
     lib.eas_encoder_destroy.restype = None
@@ -212,6 +216,20 @@ class Encoder:
     def status(self, stream=None):
         """eas_encoder_status: synchronises the stream and raises on a device-side error."""
         _check(self.lib.eas_encoder_status(self.handle, _stream_ptr(stream)))
+
+    def enable_timing(self, on: bool):
+        _check(self.lib.eas_encoder_enable_timing(self.handle, int(on)))
+
+    def timing_read(self):
+        """-> (kernel classes int32 [n], milliseconds float32 [n]) of the last timed call, in launch order."""
+        n = self.lib.eas_encoder_timing_read(self.handle, 0, None, None)
+        cls = np.zeros(max(n, 1), dtype=np.int32)
+        ms = np.zeros(max(n, 1), dtype=np.float32)
+        got = self.lib.eas_encoder_timing_read(self.handle, n, cls.ctypes.data_as(C.POINTER(C.c_int32)),
+                                               ms.ctypes.data_as(C.POINTER(C.c_float)))
+        if got < 0:
+            raise EasError(4, "timing read failed")
+        return cls[:got], ms[:got]
 
     def last_launch_count(self) -> int:
         return self.lib.eas_encoder_last_launch_count(self.handle)

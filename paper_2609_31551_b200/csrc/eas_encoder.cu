@@ -108,7 +108,28 @@ struct eas_encoder {
   int attn_impl = 0;
   int last_launches = 0;
   uint32_t* last_status = nullptr;
+  // optional per-kernel timing: one event before every launch and one after the last
+  bool timing = false;
+  std::vector<cudaEvent_t> tev;
+  std::vector<int> tcls;
+  ~eas_encoder() {
+    for (cudaEvent_t ev : tev) cudaEventDestroy(ev);
+  }
 };
+
+// records an event in front of the next launch when timing is on; cls < 0 closes the sequence
+static eas_status mark(eas_encoder* e, int cls, cudaStream_t stream) {
+  if (!e->timing) return EAS_OK;
+  const size_t i = e->tcls.size();
+  if (i >= e->tev.size()) {
+    cudaEvent_t ev;
+    CUDA_TRY(cudaEventCreate(&ev));
+    e->tev.push_back(ev);
+  }
+  CUDA_TRY(cudaEventRecord(e->tev[i], stream));
+  e->tcls.push_back(cls);
+  return EAS_OK;
+}
 
 static size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
@@ -220,10 +241,12 @@ constexpr int kOnePerSmSmem = 120 * 1024;
 static eas_status device_check(int* sm_count) {
   int dev = 0;
   CUDA_TRY(cudaGetDevice(&dev));
-  cudaDeviceProp prop;
-  CUDA_TRY(cudaGetDeviceProperties(&prop, dev));
-  if (prop.major != 10) return fail(EAS_ERR_ARCH, "device is compute capability %d.%d; this library is built for 10.x", prop.major, prop.minor);
-  *sm_count = prop.multiProcessorCount;
+  int major = 0, minor = 0, sms = 0;
+  CUDA_TRY(cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev));
+  CUDA_TRY(cudaDeviceGetAttribute(&minor, cudaDevAttrComputeCapabilityMinor, dev));
+  CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+  if (major != 10) return fail(EAS_ERR_ARCH, "device is compute capability %d.%d; this library is built for 10.x", major, minor);
+  *sm_count = sms;
   return EAS_OK;
 }
 
@@ -621,6 +644,8 @@ extern "C" eas_status eas_encode_microbatch(eas_encoder* e, const eas_packed_inp
   e->last_status = status;
 
   CUDA_TRY(cudaMemsetAsync(status, 0, 16, stream));
+  e->tcls.clear();
+  EAS_TRY(mark(e, EAS_KC_PREP, stream));
 
   // ---- tables: row maps, rotary (cos, sin), CLS rows
   {
@@ -648,6 +673,7 @@ extern "C" eas_status eas_encode_microbatch(eas_encoder* e, const eas_packed_inp
     sp.n_mel = c.in_channels; sp.d_model = d; sp.padded_rows = static_cast<int>(pl.padded_rows); sp.items = items;
     static bool attr_set = false;
     if (!attr_set) { CUDA_TRY(cudaFuncSetAttribute(audio_stage_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kOnePerSmSmem)); attr_set = true; }
+    EAS_TRY(mark(e, EAS_KC_EMBED_GATHER, stream));
     audio_stage_kernel<<<budget, 512, kOnePerSmSmem, stream>>>(sp);
     CUDA_TRY(cudaGetLastError());
     ++launches;
@@ -655,11 +681,13 @@ extern "C" eas_status eas_encode_microbatch(eas_encoder* e, const eas_packed_inp
     g1.A = mel_pad; g1.a_run = c.in_channels; g1.a_row_elems = c.in_channels; g1.conv_stride = 1; g1.taps = 3;
     g1.a_rows = pl.padded_rows; g1.M = static_cast<int>(pl.padded_rows); g1.lin = &e->conv1; g1.act = ACT_GELU;
     g1.out = h1_pad; g1.ldo = d; g1.row_map = conv1_map;
+    EAS_TRY(mark(e, EAS_KC_GEMM_EMBED, stream));
     EAS_TRY(launch_gemm(g1, budget, stream, status)); ++launches;
     GemmCall g2;   // conv2 (k=3, stride 2) + GELU + position table -> residual stream
     g2.A = h1_pad; g2.a_run = d; g2.a_row_elems = d; g2.conv_stride = 2; g2.taps = 3;
     g2.a_rows = pl.padded_rows; g2.M = static_cast<int>(pl.embed_rows); g2.lin = &e->conv2; g2.act = ACT_GELU; g2.out_fp32 = 1;
     g2.out = x; g2.ldo = d; g2.row_map = row_map; g2.pos_idx = pos_idx; g2.pos = e->pos;
+    EAS_TRY(mark(e, EAS_KC_GEMM_EMBED, stream));
     EAS_TRY(launch_gemm(g2, budget, stream, status)); ++launches;
   } else {
     Im2colParams ip{};
@@ -670,6 +698,7 @@ extern "C" eas_status eas_encode_microbatch(eas_encoder* e, const eas_packed_inp
     ip.items = items;
     static bool attr_set = false;
     if (!attr_set) { CUDA_TRY(cudaFuncSetAttribute(im2col_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kOnePerSmSmem)); attr_set = true; }
+    EAS_TRY(mark(e, EAS_KC_EMBED_GATHER, stream));
     im2col_kernel<<<budget, 512, kOnePerSmSmem, stream>>>(ip);
     CUDA_TRY(cudaGetLastError());
     ++launches;
@@ -677,10 +706,12 @@ extern "C" eas_status eas_encode_microbatch(eas_encoder* e, const eas_packed_inp
     g.A = embed_a; g.a_run = e->embed_k_pad; g.a_row_elems = e->embed_k_pad; g.a_rows = pl.embed_rows; g.M = static_cast<int>(pl.embed_rows);
     g.lin = &e->embed; g.out_fp32 = 1; g.out = x; g.ldo = d; g.row_map = row_map;
     if (c.pos == EAS_POS_TABLE) { g.pos_idx = pos_idx; g.pos = e->pos; }
+    EAS_TRY(mark(e, EAS_KC_GEMM_EMBED, stream));
     EAS_TRY(launch_gemm(g, budget, stream, status)); ++launches;
   }
   if (c.embed_norm) {
     NormParams np{x, x, e->eng, e->enb, nullptr, static_cast<int>(T), d, c.norm_eps};
+    EAS_TRY(mark(e, EAS_KC_NORM, stream));
     EAS_TRY(launch_norm(ln_kind, true, np, budget, stream)); ++launches;
   }
 
@@ -689,6 +720,7 @@ extern "C" eas_status eas_encode_microbatch(eas_encoder* e, const eas_packed_inp
     const Layer& L = e->layers[li];
     {
       NormParams np{x, nbuf, L.n1g, L.n1b, nullptr, static_cast<int>(T), d, c.norm_eps};
+      EAS_TRY(mark(e, EAS_KC_NORM, stream));
       EAS_TRY(launch_norm(ln_kind, false, np, budget, stream)); ++launches;
     }
     {
@@ -696,17 +728,21 @@ extern "C" eas_status eas_encode_microbatch(eas_encoder* e, const eas_packed_inp
       g.A = nbuf; g.a_run = d; g.a_row_elems = d; g.a_rows = T; g.M = static_cast<int>(T); g.lin = &L.qkv;
       g.out = qkv; g.ldo = 3LL * d;
       if (c.pos == EAS_POS_ROPE_2D) { g.rope_cs = rope; g.rope_pairs = e->hd / 2; g.rope_ncols = 2 * d; g.head_dim = e->hd; }
+      EAS_TRY(mark(e, EAS_KC_GEMM_QKV, stream));
       EAS_TRY(launch_gemm(g, budget, stream, status)); ++launches;
     }
+    EAS_TRY(mark(e, EAS_KC_ATTENTION, stream));
     EAS_TRY(launch_attention(qkv, obuf, cu, n, c.n_heads, e->hd, budget, stream, e->attn_impl, status)); ++launches;
     {
       GemmCall g;
       g.A = obuf; g.a_run = d; g.a_row_elems = d; g.a_rows = T; g.M = static_cast<int>(T); g.lin = &L.proj;
       g.out_fp32 = 1; g.out = x; g.ldo = d; g.resid = x;
+      EAS_TRY(mark(e, EAS_KC_GEMM_PROJ, stream));
       EAS_TRY(launch_gemm(g, budget, stream, status)); ++launches;
     }
     {
       NormParams np{x, nbuf, L.n2g, L.n2b, nullptr, static_cast<int>(T), d, c.norm_eps};
+      EAS_TRY(mark(e, EAS_KC_NORM, stream));
       EAS_TRY(launch_norm(ln_kind, false, np, budget, stream)); ++launches;
     }
     {
@@ -714,17 +750,20 @@ extern "C" eas_status eas_encode_microbatch(eas_encoder* e, const eas_packed_inp
       g.A = nbuf; g.a_run = d; g.a_row_elems = d; g.a_rows = T; g.M = static_cast<int>(T); g.lin = &L.fc1;
       g.act = c.mlp == EAS_MLP_SWIGLU ? ACT_SWIGLU : ACT_GELU;
       g.out = abuf; g.ldo = c.d_mlp;
+      EAS_TRY(mark(e, EAS_KC_GEMM_FC1, stream));
       EAS_TRY(launch_gemm(g, budget, stream, status)); ++launches;
     }
     {
       GemmCall g;
       g.A = abuf; g.a_run = c.d_mlp; g.a_row_elems = c.d_mlp; g.a_rows = T; g.M = static_cast<int>(T); g.lin = &L.fc2;
       g.out_fp32 = 1; g.out = x; g.ldo = d; g.resid = x;
+      EAS_TRY(mark(e, EAS_KC_GEMM_FC2, stream));
       EAS_TRY(launch_gemm(g, budget, stream, status)); ++launches;
     }
   }
 
   // ---- connector
+  EAS_TRY(mark(e, EAS_KC_NORM, stream));
   if (c.head == EAS_HEAD_NONE) {
     if (c.final_norm) {
       NormParams np{x, out_embeddings, e->fng, e->fnb, nullptr, static_cast<int>(T), d, c.norm_eps};
@@ -749,14 +788,37 @@ extern "C" eas_status eas_encode_microbatch(eas_encoder* e, const eas_packed_inp
     GemmCall g1;
     g1.A = nbuf; g1.a_run = k_in; g1.a_row_elems = k_in; g1.a_rows = rows_in; g1.M = static_cast<int>(rows_in); g1.lin = &e->head1;
     g1.act = ACT_GELU; g1.out = abuf; g1.ldo = c.d_head_hidden;
+    EAS_TRY(mark(e, EAS_KC_GEMM_HEAD, stream));
     EAS_TRY(launch_gemm(g1, budget, stream, status)); ++launches;
     GemmCall g2;
     g2.A = abuf; g2.a_run = c.d_head_hidden; g2.a_row_elems = c.d_head_hidden; g2.a_rows = rows_in; g2.M = static_cast<int>(rows_in); g2.lin = &e->head2;
     g2.out = out_embeddings; g2.ldo = c.d_out;
+    EAS_TRY(mark(e, EAS_KC_GEMM_HEAD, stream));
     EAS_TRY(launch_gemm(g2, budget, stream, status)); ++launches;
   }
+  EAS_TRY(mark(e, -1, stream));
   e->last_launches = launches;
   return EAS_OK;
+}
+
+extern "C" eas_status eas_encoder_enable_timing(eas_encoder* e, int32_t on) {
+  if (e == nullptr) return fail(EAS_ERR_INVALID_ARG, "encoder is null");
+  e->timing = on != 0;
+  e->tcls.clear();
+  return EAS_OK;
+}
+
+extern "C" int32_t eas_encoder_timing_read(eas_encoder* e, int32_t capacity, int32_t* kernel_class, float* ms) {
+  if (e == nullptr || e->tcls.size() < 2) return 0;
+  const int n = static_cast<int>(e->tcls.size()) - 1;
+  if (kernel_class == nullptr || ms == nullptr) return n;
+  if (cudaEventSynchronize(e->tev[n]) != cudaSuccess) return -1;
+  const int m = std::min(n, capacity);
+  for (int i = 0; i < m; ++i) {
+    kernel_class[i] = e->tcls[i];
+    if (cudaEventElapsedTime(&ms[i], e->tev[i], e->tev[i + 1]) != cudaSuccess) return -1;
+  }
+  return m;
 }
 
 extern "C" eas_status eas_encoder_status(eas_encoder* e, void* stream_v) {
@@ -791,7 +853,8 @@ extern "C" eas_status eas_kernel_gemm(const void* A, const void* W, const void* 
   if (act < 0 || act > 2 || (act == ACT_SWIGLU && out_fp32)) return fail(EAS_ERR_INVALID_ARG, "bad epilogue selection");
   int budget = 0;
   EAS_TRY(resolve_budget(sm_budget, &budget));
-  EAS_TRY(set_kernel_attributes());
+  static bool attrs_done = false;
+  if (!attrs_done) { EAS_TRY(set_kernel_attributes()); attrs_done = true; }
   Linear L;
   L.w = static_cast<const bf16*>(W); L.b = static_cast<const bf16*>(bias); L.N = N; L.K = K;
   EAS_TRY(finish_linear(L));
