@@ -1,0 +1,390 @@
+// Block-diagonal (variable-length) softmax attention on tcgen05 tensor cores.
+//
+// One work unit = (item, head, 256 query rows) = two 128-row query tiles A and B that share every
+// K/V tile.  Keys and values come from the same item only: the key loop stops at the item's last
+// 128-key tile and the keys past the item's end are masked to -inf (probability exactly 0).
+//
+//   warp 0       TMA producer: Q tiles (double buffered across units), K/V tiles through a ring
+//   warp 1       UMMA issuer:  S = Q K^T (128x128x{64|80}) into TMEM, O += P V (128x{64|80}x128) in TMEM
+//   warps 2..5   softmax warpgroup of tile A: one thread per query row
+//   warps 6..9   softmax warpgroup of tile B
+//
+// A softmax thread reads its row of S from TMEM, keeps a running reference maximum m and sum l, writes
+// P = exp2((s - m) * scale) as bf16 into shared memory (K-major, 128-byte swizzle: the A operand of P V).
+// The reference maximum only moves when the row maximum grows by more than 2^8 in the exponent; then the
+// thread rescales its O row in TMEM.  Final O / l is written as bf16.
+// Persistent: gridDim.x = sm_budget CTAs walk units blockIdx.x, +gridDim.x, ... in a fixed order.
+#pragma once
+#include "ptx.cuh"
+
+namespace eas {
+
+constexpr int kTcThreads = 320;
+constexpr int kTcTile = 128;            // query rows per tile and keys per K/V tile
+constexpr float kRescaleThreshold = 8.0f;
+
+struct AttnTcParams {
+  CUtensorMap map_lo;   // qkv [T, 3d], box {64 columns, 128 rows}, 128-byte swizzle
+  CUtensorMap map_hi;   // box {16 columns, 128 rows}, 32-byte swizzle (head_dim 80: columns 64..79)
+  bf16* out;
+  long long ldo;
+  int d_model, n_heads;
+  float scale_log2;     // log2(e) / sqrt(head_dim)
+  int n_items, total_units;
+  int item_start[128];
+  int item_len[128];
+  int unit_prefix[129];
+  uint32_t* status;
+};
+
+template <int HD>
+struct AttnTcSmem {
+  static constexpr int HI = HD - 64;                       // 0 or 16 extra columns
+  static constexpr int kLoBytes = kTcTile * 128;           // 128 rows x 64 bf16
+  static constexpr int kHiBytes = kTcTile * HI * 2;        // 128 rows x 16 bf16
+  static constexpr int kTileBytes = kLoBytes + kHiBytes;   // one Q, K or V tile
+  static constexpr int kStages = HD == 64 ? 3 : 2;
+  static constexpr int kQOff = 0;                          // [2 buffers][2 tiles]
+  static constexpr int kKvOff = kQOff + 4 * kTileBytes;    // [stages][K, V]
+  static constexpr int kPOff = kKvOff + kStages * 2 * kTileBytes;   // [2 tiles][2 k-blocks of 16 KB]
+  static constexpr int kBarOff = kPOff + 2 * 32768;
+  static constexpr int kBytes = kBarOff + 512 + 1024;      // barriers + alignment slack
+};
+
+__device__ __forceinline__ void tmem_ld_32x16(uint32_t taddr, uint32_t (&r)[16]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_st_32x16(uint32_t taddr, const uint32_t (&r)[16]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
+      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
+      ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+        "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
+      : "memory");
+}
+__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+struct UnitInfo {
+  int head, q0, S, n_kv, n_q;
+  long long row0;
+};
+__device__ __forceinline__ UnitInfo decode_unit(const AttnTcParams& p, int unit) {
+  int lo = 0, hi = p.n_items - 1;
+  while (lo < hi) {
+    const int mid = (lo + hi + 1) >> 1;
+    if (p.unit_prefix[mid] <= unit) lo = mid; else hi = mid - 1;
+  }
+  UnitInfo u;
+  u.S = p.item_len[lo];
+  u.row0 = p.item_start[lo];
+  const int pairs = (u.S + 2 * kTcTile - 1) / (2 * kTcTile);
+  const int r = unit - p.unit_prefix[lo];
+  u.head = r / pairs;
+  u.q0 = (r - u.head * pairs) * 2 * kTcTile;       // pair index varies fastest: neighbours share K and V in L2
+  u.n_kv = (u.S + kTcTile - 1) / kTcTile;
+  u.n_q = (u.q0 + kTcTile < u.S) ? 2 : 1;
+  return u;
+}
+
+template <int HD>
+__global__ void __launch_bounds__(kTcThreads, 1) attn_tc_kernel(const __grid_constant__ AttnTcParams p) {
+  using L = AttnTcSmem<HD>;
+  constexpr int HI = L::HI;
+  constexpr int NST = L::kStages;
+  extern __shared__ uint8_t smem_raw_attn[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw_attn) + 1023) & ~uintptr_t(1023));
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L::kBarOff);
+  uint64_t* q_full = bars;                 // [2]
+  uint64_t* q_empty = bars + 2;            // [2]
+  uint64_t* k_full = bars + 4;             // [NST]
+  uint64_t* v_full = bars + 4 + NST;       // [NST]
+  uint64_t* kv_empty = bars + 4 + 2 * NST; // [NST]
+  uint64_t* s_full = bars + 4 + 3 * NST;   // [2]
+  uint64_t* p_ready = s_full + 2;          // [2]
+  uint64_t* pv_done = s_full + 4;          // [2]
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(s_full + 6);
+  volatile uint32_t* abort_flag = tmem_slot + 1;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(&q_full[i], 1); mbar_init(&q_empty[i], 1);
+      mbar_init(&s_full[i], 1); mbar_init(&p_ready[i], 4); mbar_init(&pv_done[i], 1);
+    }
+    for (int i = 0; i < NST; ++i) { mbar_init(&k_full[i], 1); mbar_init(&v_full[i], 1); mbar_init(&kv_empty[i], 1); }
+    *abort_flag = 0;
+    mbar_fence_init();
+    tma_prefetch_desc(&p.map_lo);
+    if (HI) tma_prefetch_desc(&p.map_hi);
+  }
+  if (warp == 1) {
+    tmem_alloc(tmem_slot, 512);
+    tmem_relinquish();
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem_base = *tmem_slot;
+  // TMEM columns: S_A [0,128)  S_B [128,256)  O_A [256,256+HD)  O_B [384,384+HD)
+
+  auto q_tile = [&](int buf, int t) { return smem + L::kQOff + (buf * 2 + t) * L::kTileBytes; };
+  auto k_tile = [&](int s) { return smem + L::kKvOff + (s * 2) * L::kTileBytes; };
+  auto v_tile = [&](int s) { return smem + L::kKvOff + (s * 2 + 1) * L::kTileBytes; };
+  auto p_tile = [&](int w) { return smem + L::kPOff + w * 32768; };
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      uint32_t kv_it = 0, u_cnt = 0;
+      bool ok = true;
+      for (int unit = blockIdx.x; unit < p.total_units && ok; unit += gridDim.x, ++u_cnt) {
+        const UnitInfo u = decode_unit(p, unit);
+        const int qb = u_cnt & 1;
+        if (!mbar_wait(&q_empty[qb], ((u_cnt >> 1) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+        mbar_expect_tx(&q_full[qb], u.n_q * L::kTileBytes);
+        const int xq = u.head * HD;
+        for (int t = 0; t < u.n_q; ++t) {
+          const int y = static_cast<int>(u.row0) + u.q0 + t * kTcTile;
+          tma_load_2d(q_tile(qb, t), &p.map_lo, &q_full[qb], xq, y);
+          if (HI) tma_load_2d(q_tile(qb, t) + L::kLoBytes, &p.map_hi, &q_full[qb], xq + 64, y);
+        }
+        for (int j = 0; j < u.n_kv; ++j, ++kv_it) {
+          const int s = kv_it % NST;
+          if (!mbar_wait(&kv_empty[s], ((kv_it / NST) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+          const int y = static_cast<int>(u.row0) + j * kTcTile;
+          mbar_expect_tx(&k_full[s], L::kTileBytes);
+          tma_load_2d(k_tile(s), &p.map_lo, &k_full[s], p.d_model + xq, y);
+          if (HI) tma_load_2d(k_tile(s) + L::kLoBytes, &p.map_hi, &k_full[s], p.d_model + xq + 64, y);
+          mbar_expect_tx(&v_full[s], L::kTileBytes);
+          tma_load_2d(v_tile(s), &p.map_lo, &v_full[s], 2 * p.d_model + xq, y);
+          if (HI) tma_load_2d(v_tile(s) + L::kLoBytes, &p.map_hi, &v_full[s], 2 * p.d_model + xq + 64, y);
+        }
+      }
+      if (!ok) {
+        const long long t0 = clock64();
+        while (clock64() - t0 < 4000000) {}     // let loads in flight land before the CTA retires
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ UMMA issuer
+    if (lane == 0) {
+      constexpr uint32_t idesc_s = make_idesc_bf16(128, 128, 0, 0);     // S = Q K^T, both K-major
+      constexpr uint32_t idesc_o_lo = make_idesc_bf16(128, 64, 0, 1);   // O[:, 0:64] += P V, V is MN-major
+      constexpr uint32_t idesc_o_hi = make_idesc_bf16(128, 16, 0, 1);   // O[:, 64:80]
+      uint32_t kv_it = 0, u_cnt = 0;
+      uint32_t n_tiles[2] = {0, 0};            // S tiles issued per warpgroup (phase counters)
+      uint32_t n_pv[2] = {0, 0};
+      bool ok = true;
+
+      auto issue_s = [&](int w, int qb, int s) {
+        const uint32_t qa = smem_u32(q_tile(qb, w));
+        const uint32_t ka = smem_u32(k_tile(s));
+        const uint64_t ad = make_smem_desc(qa, 16, 1024, kSwizzle128B);
+        const uint64_t bd = make_smem_desc(ka, 16, 1024, kSwizzle128B);
+        const uint32_t d = tmem_base + w * 128;
+#pragma unroll
+        for (int k = 0; k < 4; ++k) umma_bf16_ss(d, ad + 2 * k, bd + 2 * k, idesc_s, k != 0);
+        if (HI) {
+          const uint64_t ah = make_smem_desc(qa + L::kLoBytes, 16, 256, kSwizzle32B);
+          const uint64_t bh = make_smem_desc(ka + L::kLoBytes, 16, 256, kSwizzle32B);
+          umma_bf16_ss(d, ah, bh, idesc_s, 1);
+        }
+        umma_commit(&s_full[w]);
+        ++n_tiles[w];
+      };
+      auto issue_pv = [&](int w, int s, bool accumulate) {
+        const uint32_t pa = smem_u32(p_tile(w));
+        const uint32_t va = smem_u32(v_tile(s));
+        const uint32_t d = tmem_base + 256 + w * 128;
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks) {       // 16 keys per step
+          const uint64_t ad = make_smem_desc(pa + (ks >> 2) * 16384 + (ks & 3) * 32, 16, 1024, kSwizzle128B);
+          const uint64_t bd = make_smem_desc(va + ks * 2048, 1024, 1024, kSwizzle128B);
+          umma_bf16_ss(d, ad, bd, idesc_o_lo, (accumulate || ks != 0) ? 1u : 0u);
+          if (HI) {
+            const uint64_t bh = make_smem_desc(va + L::kLoBytes + ks * 512, 256, 256, kSwizzle32B);
+            umma_bf16_ss(d + 64, ad, bh, idesc_o_hi, (accumulate || ks != 0) ? 1u : 0u);
+          }
+        }
+        umma_commit(&pv_done[w]);
+        ++n_pv[w];
+      };
+
+      for (int unit = blockIdx.x; unit < p.total_units && ok; unit += gridDim.x, ++u_cnt) {
+        const UnitInfo u = decode_unit(p, unit);
+        const int qb = u_cnt & 1;
+        if (!mbar_wait(&q_full[qb], (u_cnt >> 1) & 1u, abort_flag)) { ok = false; break; }
+        {
+          const int s = kv_it % NST;
+          if (!mbar_wait(&k_full[s], (kv_it / NST) & 1u, abort_flag)) { ok = false; break; }
+          tc_fence_after_sync();
+          for (int w = 0; w < u.n_q; ++w) issue_s(w, qb, s);
+        }
+        for (int j = 0; j < u.n_kv && ok; ++j, ++kv_it) {
+          const int s = kv_it % NST;
+          const int sn = (kv_it + 1) % NST;
+          for (int w = 0; w < u.n_q; ++w) {
+            // P(w, j) is in shared memory, S(w) has been read, O(w) has been rescaled if it had to be
+            if (!mbar_wait(&p_ready[w], (n_pv[w]) & 1u, abort_flag)) { ok = false; break; }
+            tc_fence_after_sync();
+            if (j + 1 < u.n_kv) {
+              if (w == 0 && !mbar_wait(&k_full[sn], ((kv_it + 1) / NST) & 1u, abort_flag)) { ok = false; break; }
+              tc_fence_after_sync();
+              issue_s(w, qb, sn);              // next scores first: the softmax of tile j+1 overlaps P V of tile j
+            }
+            if (w == 0 && !mbar_wait(&v_full[s], (kv_it / NST) & 1u, abort_flag)) { ok = false; break; }
+            tc_fence_after_sync();
+            issue_pv(w, s, j != 0);
+          }
+          if (ok) umma_commit(&kv_empty[s]);   // K(j) and V(j) are free once everything issued so far completes
+        }
+        if (ok) umma_commit(&q_empty[qb]);
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ softmax warpgroups
+    const int w = (warp - 2) >> 2;                 // 0: tile A, 1: tile B
+    const int quarter = warp & 3;                  // TMEM lane quarter of this warp
+    const int row = quarter * 32 + lane;           // query row inside the tile == TMEM lane
+    const uint32_t lane_addr = static_cast<uint32_t>(quarter * 32) << 16;
+    const uint32_t s_addr = tmem_base + lane_addr + w * 128;
+    const uint32_t o_addr = tmem_base + lane_addr + 256 + w * 128;
+    uint8_t* p_row = p_tile(w) + row * 128;
+    const int sw = row & 7;
+    uint32_t n = 0;                                // tiles processed by this warpgroup
+    bool ok = true;
+
+    for (int unit = blockIdx.x; unit < p.total_units && ok; unit += gridDim.x) {
+      const UnitInfo u = decode_unit(p, unit);
+      if (w >= u.n_q) continue;
+      float m_used = -INFINITY, l = 0.f;
+      for (int j = 0; j < u.n_kv; ++j, ++n) {
+        if (!mbar_wait(&s_full[w], n & 1u, abort_flag)) { ok = false; break; }
+        tc_fence_after_sync();
+        const int valid = min(kTcTile, u.S - j * kTcTile);     // keys of this tile that belong to the item
+        // pass 1: row maximum
+        float mx = -INFINITY;
+#pragma unroll 1
+        for (int c = 0; c < 4; ++c) {
+          uint32_t raw[32];
+          __syncwarp();
+          tmem_ld_32x32(s_addr + c * 32, raw);
+          tmem_ld_wait();
+          if (valid >= (c + 1) * 32) {
+#pragma unroll
+            for (int i = 0; i < 32; ++i) mx = fmaxf(mx, __uint_as_float(raw[i]));
+          } else {
+#pragma unroll
+            for (int i = 0; i < 32; ++i) if (c * 32 + i < valid) mx = fmaxf(mx, __uint_as_float(raw[i]));
+          }
+        }
+        // reference maximum: moves only when the row maximum grew by more than the threshold
+        float corr = 1.0f;
+        bool rescale = false;
+        if (j == 0) {
+          m_used = mx;
+        } else if ((mx - m_used) * p.scale_log2 > kRescaleThreshold) {
+          corr = fast_ex2((m_used - mx) * p.scale_log2);
+          m_used = mx;
+          rescale = true;
+        }
+        l *= corr;
+        const float mb = m_used * p.scale_log2;
+        // pass 2: probabilities, kept packed in registers until the P buffer is free
+        uint32_t pk[64];
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          uint32_t raw[32];
+          __syncwarp();
+          tmem_ld_32x32(s_addr + c * 32, raw);
+          tmem_ld_wait();
+          float sum = 0.f;
+#pragma unroll
+          for (int i = 0; i < 32; i += 2) {
+            float p0 = fast_ex2(fmaf(__uint_as_float(raw[i]), p.scale_log2, -mb));
+            float p1 = fast_ex2(fmaf(__uint_as_float(raw[i + 1]), p.scale_log2, -mb));
+            if (c * 32 + i >= valid) p0 = 0.f;
+            if (c * 32 + i + 1 >= valid) p1 = 0.f;
+            sum += p0 + p1;
+            pk[c * 16 + (i >> 1)] = pack_bf16x2(p0, p1);
+          }
+          l += sum;
+        }
+        // S has been read: the issuer may overwrite it with the next tile's scores once p_ready fires.
+        // The previous P V must be complete before P is overwritten or O is touched.
+        if (n > 0 && !mbar_wait(&pv_done[w], (n - 1) & 1u, abort_flag)) { ok = false; break; }
+        tc_fence_after_sync();
+        if (__any_sync(0xffffffffu, rescale)) {
+#pragma unroll 1
+          for (int c = 0; c < HD / 16; ++c) {
+            uint32_t o[16];
+            __syncwarp();
+            tmem_ld_32x16(o_addr + c * 16, o);
+            tmem_ld_wait();
+#pragma unroll
+            for (int i = 0; i < 16; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * corr);
+            tmem_st_32x16(o_addr + c * 16, o);
+          }
+          tmem_st_wait();
+        }
+        // P row: 2 k-blocks of 64 keys, each row 128 bytes, 16-byte chunks XOR-swizzled by (row & 7)
+#pragma unroll
+        for (int cc = 0; cc < 16; ++cc) {
+          const int kblk = cc >> 3, ch = cc & 7;
+          uint4 v = make_uint4(pk[cc * 4], pk[cc * 4 + 1], pk[cc * 4 + 2], pk[cc * 4 + 3]);
+          *reinterpret_cast<uint4*>(p_row + kblk * 16384 + ((ch ^ sw) << 4)) = v;
+        }
+        fence_proxy_async_smem();
+        tc_fence_before_sync();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&p_ready[w]);
+      }
+      if (!ok) break;
+      // epilogue: O / l -> bf16
+      if (!mbar_wait(&pv_done[w], (n - 1) & 1u, abort_flag)) { ok = false; break; }
+      tc_fence_after_sync();
+      const float inv = 1.0f / l;
+      const int qrow = u.q0 + w * kTcTile + row;
+      bf16* orow = p.out + (u.row0 + qrow) * p.ldo + u.head * HD;
+#pragma unroll 1
+      for (int c = 0; c < HD / 16; ++c) {
+        uint32_t o[16];
+        __syncwarp();
+        tmem_ld_32x16(o_addr + c * 16, o);
+        tmem_ld_wait();
+        if (qrow < u.S) {
+          uint4 v0 = make_uint4(pack_bf16x2(__uint_as_float(o[0]) * inv, __uint_as_float(o[1]) * inv),
+                                pack_bf16x2(__uint_as_float(o[2]) * inv, __uint_as_float(o[3]) * inv),
+                                pack_bf16x2(__uint_as_float(o[4]) * inv, __uint_as_float(o[5]) * inv),
+                                pack_bf16x2(__uint_as_float(o[6]) * inv, __uint_as_float(o[7]) * inv));
+          uint4 v1 = make_uint4(pack_bf16x2(__uint_as_float(o[8]) * inv, __uint_as_float(o[9]) * inv),
+                                pack_bf16x2(__uint_as_float(o[10]) * inv, __uint_as_float(o[11]) * inv),
+                                pack_bf16x2(__uint_as_float(o[12]) * inv, __uint_as_float(o[13]) * inv),
+                                pack_bf16x2(__uint_as_float(o[14]) * inv, __uint_as_float(o[15]) * inv));
+          uint4* dst = reinterpret_cast<uint4*>(orow + c * 16);
+          dst[0] = v0;
+          dst[1] = v1;
+        }
+      }
+      // the O reads above must complete before this warpgroup's next p_ready lets P V overwrite O
+      tc_fence_before_sync();
+    }
+  }
+
+  tc_fence_before_sync();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after_sync();
+    tmem_dealloc(tmem_base, 512);
+  }
+  if (threadIdx.x == 0 && *abort_flag) atomicCAS(p.status, DEV_OK, DEV_ERR_WAIT_TIMEOUT);
+}
+
+}  // namespace eas

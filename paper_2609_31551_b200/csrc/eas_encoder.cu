@@ -17,6 +17,7 @@
 #include <vector>
 
 #include "attention_mma.cuh"
+#include "attention_tc.cuh"
 #include "elementwise.cuh"
 #include "gemm.cuh"
 
@@ -530,29 +531,34 @@ static eas_status launch_norm(int kind, bool out_fp32, const NormParams& p, int 
   return fail(EAS_ERR_INVALID_ARG, "unknown norm kind %d", kind);
 }
 
-static eas_status launch_attention(const bf16* qkv, bf16* out, const int32_t* cu, int n_items, int H, int hd, int budget,
-                                   cudaStream_t stream, int /*impl*/, uint32_t* /*status*/) {
-  AttnParams ap{};
-  const int d = H * hd;
-  ap.qkv = qkv; ap.out = out; ap.ld = 3LL * d; ap.ldo = d; ap.d_model = d; ap.n_heads = H;
-  ap.scale_log2 = static_cast<float>(1.4426950408889634 / std::sqrt(static_cast<double>(hd)));
-  ap.n_items = n_items;
-  // schedule order: longest items first (stable), so the tail of the static round-robin is short work
+// schedule order: longest items first (stable), so the tail of the static round-robin is short work
+static void attention_schedule(const int32_t* cu, int n_items, int rows_per_unit, int H, int* item_start, int* item_len,
+                               int* unit_prefix, int* total_units) {
   std::vector<int> order(n_items);
   for (int i = 0; i < n_items; ++i) order[i] = i;
   std::stable_sort(order.begin(), order.end(), [&](int a, int b) { return (cu[a + 1] - cu[a]) > (cu[b + 1] - cu[b]); });
   int units = 0;
   for (int k = 0; k < n_items; ++k) {
     const int i = order[k];
-    ap.item_start[k] = cu[i];
-    ap.item_len[k] = cu[i + 1] - cu[i];
-    ap.unit_prefix[k] = units;
-    units += ((ap.item_len[k] + kAttnBQ - 1) / kAttnBQ) * H;
+    item_start[k] = cu[i];
+    item_len[k] = cu[i + 1] - cu[i];
+    unit_prefix[k] = units;
+    units += ((item_len[k] + rows_per_unit - 1) / rows_per_unit) * H;
   }
-  ap.unit_prefix[n_items] = units;
-  ap.total_units = units;
-  if (units == 0) return EAS_OK;
-  const int grid = std::min(budget, units);
+  unit_prefix[n_items] = units;
+  *total_units = units;
+}
+
+static eas_status launch_attention_mma(const bf16* qkv, bf16* out, const int32_t* cu, int n_items, int H, int hd, int budget,
+                                       cudaStream_t stream) {
+  AttnParams ap{};
+  const int d = H * hd;
+  ap.qkv = qkv; ap.out = out; ap.ld = 3LL * d; ap.ldo = d; ap.d_model = d; ap.n_heads = H;
+  ap.scale_log2 = static_cast<float>(1.4426950408889634 / std::sqrt(static_cast<double>(hd)));
+  ap.n_items = n_items;
+  attention_schedule(cu, n_items, kAttnBQ, H, ap.item_start, ap.item_len, ap.unit_prefix, &ap.total_units);
+  if (ap.total_units == 0) return EAS_OK;
+  const int grid = std::min(budget, ap.total_units);
   static bool attr_set = false;
   if (!attr_set) {
     CUDA_TRY(cudaFuncSetAttribute(attn_mma_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, kOnePerSmSmem));
@@ -565,6 +571,45 @@ static eas_status launch_attention(const bf16* qkv, bf16* out, const int32_t* cu
   else return fail(EAS_ERR_UNSUPPORTED, "head_dim %d", hd);
   CUDA_TRY(cudaGetLastError());
   return EAS_OK;
+}
+
+static eas_status launch_attention_tc(const bf16* qkv, bf16* out, const int32_t* cu, int n_items, int H, int hd, int budget,
+                                      cudaStream_t stream, uint32_t* status) {
+  AttnTcParams ap{};
+  const int d = H * hd;
+  const int64_t T = cu[n_items];
+  {
+    const uint64_t dims[2] = {static_cast<uint64_t>(3 * d), static_cast<uint64_t>(T)};
+    const uint64_t strides[1] = {static_cast<uint64_t>(3 * d) * 2};
+    const uint32_t box_lo[2] = {64, kTcTile};
+    EAS_TRY(make_tmap(&ap.map_lo, qkv, 2, dims, strides, box_lo, CU_TENSOR_MAP_SWIZZLE_128B));
+    const uint32_t box_hi[2] = {16, kTcTile};
+    EAS_TRY(make_tmap(&ap.map_hi, qkv, 2, dims, strides, box_hi, CU_TENSOR_MAP_SWIZZLE_32B));
+  }
+  ap.out = out; ap.ldo = d; ap.d_model = d; ap.n_heads = H;
+  ap.scale_log2 = static_cast<float>(1.4426950408889634 / std::sqrt(static_cast<double>(hd)));
+  ap.n_items = n_items;
+  ap.status = status;
+  attention_schedule(cu, n_items, 2 * kTcTile, H, ap.item_start, ap.item_len, ap.unit_prefix, &ap.total_units);
+  if (ap.total_units == 0) return EAS_OK;
+  const int grid = std::min(budget, ap.total_units);
+  static bool attr_set = false;
+  if (!attr_set) {
+    CUDA_TRY(cudaFuncSetAttribute(attn_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttnTcSmem<64>::kBytes));
+    CUDA_TRY(cudaFuncSetAttribute(attn_tc_kernel<80>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttnTcSmem<80>::kBytes));
+    attr_set = true;
+  }
+  if (hd == 64) attn_tc_kernel<64><<<grid, kTcThreads, AttnTcSmem<64>::kBytes, stream>>>(ap);
+  else if (hd == 80) attn_tc_kernel<80><<<grid, kTcThreads, AttnTcSmem<80>::kBytes, stream>>>(ap);
+  else return fail(EAS_ERR_UNSUPPORTED, "head_dim %d", hd);
+  CUDA_TRY(cudaGetLastError());
+  return EAS_OK;
+}
+
+static eas_status launch_attention(const bf16* qkv, bf16* out, const int32_t* cu, int n_items, int H, int hd, int budget,
+                                   cudaStream_t stream, int impl, uint32_t* status) {
+  if (impl == 1) return launch_attention_mma(qkv, out, cu, n_items, H, hd, budget, stream);
+  return launch_attention_tc(qkv, out, cu, n_items, H, hd, budget, stream, status);
 }
 
 // ------------------------------------------------------------------------------------ the forward pass
