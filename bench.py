@@ -164,19 +164,16 @@ def run_reference(args):
 # ------------------------------------------------------------------ CUDA arm
 def run_cuda(args):
     import torch
-    import torch.distributed as dist
     import paper_2609_31551_b200 as P
+    from paper_2609_31551_b200 import replicas as R
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world, rank, local_rank = R.world()
     if not torch.cuda.is_available():
         raise RuntimeError("bench.py needs a CUDA device: the encoder has no CPU fallback")
     torch.cuda.set_device(local_rank)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    R.init("nccl", torch.device("cuda", local_rank))
 
-    cfg, shapes, seed = workload(args.config, args.micro_batch, seed_shift=1000 * rank)
+    cfg, shapes, seed = workload(args.config, args.micro_batch, seed_shift=R.rank_seed_shift(rank))
     w = S.make_weights(cfg)
     enc = P.Encoder(cfg, P.weights_to_device(w))
     items = S.make_items(cfg, shapes, seed)
@@ -194,9 +191,8 @@ def run_cuda(args):
 
     def barrier():
         torch.cuda.synchronize()
-        if world > 1:
-            dist.barrier()
-            torch.cuda.synchronize()
+        R.barrier()
+        torch.cuda.synchronize()
 
     for _ in range(max(args.warmup, 3)):
         step()
@@ -273,18 +269,9 @@ def run_cuda(args):
     enc.enable_timing(False)
     torch.cuda.synchronize()
 
-    if world > 1:
-        t = torch.tensor([ms, ms_e2e], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms, ms_e2e = t.tolist()
-        tok = torch.tensor([float(T)], dtype=torch.float64, device="cuda")
-        dist.all_reduce(tok)
-        total_tokens = tok.item()
-        nl = torch.tensor([float(launches)], dtype=torch.float64, device="cuda")
-        dist.all_reduce(nl)
-        launches = int(nl.item())
-    else:
-        total_tokens = float(T)
+    (ms, ms_e2e), (total_tokens, launches, total_items, total_flops) = R.combine(
+        [ms, ms_e2e], [float(T), float(launches), float(len(shapes)), float(f["total"])], device="cuda")
+    launches = int(launches)
 
     if rank == 0:
         peaks = measured_peaks()
@@ -311,8 +298,8 @@ def run_cuda(args):
                        "tokens_per_step": T, "sm_budget": budget if budget else "all",
                        "l2": "working set (weights + activations) larger than L2; no flush",
                        "parallelism": "replicas" if world > 1 else "single"},
-            "items_per_sec": len(shapes) * world * args.steps / (ms * 1e-3),
-            "tflops": f["total"] * world / (step_ms * 1e-3) / 1e12,
+            "items_per_sec": total_items * args.steps / (ms * 1e-3),
+            "tflops": total_flops / (step_ms * 1e-3) / 1e12,
             "frac_of_bf16_peak": {"burst_measured": f["total"] / (step_ms * 1e-3) / 1e12 / peaks["burst"],
                                   "sustained_measured": f["total"] / (step_ms * 1e-3) / 1e12 / peaks["sustained"],
                                   "source": peaks["source"]},
@@ -329,8 +316,7 @@ def run_cuda(args):
         if world == 1 and not args.no_cpu_baseline:
             line["cpu_baseline"] = cpu_baseline(cfg, w, shapes, seed)
         print(json.dumps(line))
-    if world > 1:
-        dist.destroy_process_group()
+    R.finish()
 
 
 def cpu_baseline(cfg, w, shapes, seed):

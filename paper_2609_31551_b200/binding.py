@@ -199,15 +199,18 @@ class Encoder:
         T = int(cu[-1])
         need = self.workspace_bytes(T, n)
         if workspace is None:
-            if self._workspace is None or self._workspace.numel() < need:
-                self._workspace = torch.empty(max(need, 1024), dtype=torch.uint8, device=data.device)
+            if self._workspace is None or self._workspace.numel() < need + 1024:
+                self._workspace = torch.empty(need + 1024, dtype=torch.uint8, device=data.device)
             workspace = self._workspace
+        # the library wants a 1024-byte aligned workspace; small torch allocations are only 512-byte aligned
+        ws_ptr = (workspace.data_ptr() + 1023) // 1024 * 1024
+        ws_bytes = workspace.numel() - (ws_ptr - workspace.data_ptr())
         if out is None:
             rows = self.out_rows(cu)
             out = torch.empty((max(rows, 0), self.cfg["d_out"]), dtype=torch.bfloat16, device=data.device)
         pin = PackedInputs(data.data_ptr(), n, shp.ctypes.data_as(C.POINTER(C.c_int32)),
                            offs.ctypes.data_as(C.POINTER(C.c_int64)), cu.ctypes.data_as(C.POINTER(C.c_int32)),
-                           workspace.data_ptr(), workspace.numel())
+                           ws_ptr, ws_bytes)
         _check(self.lib.eas_encode_microbatch(self.handle, C.byref(pin), cu_seqlens_dev.data_ptr(), sm_budget,
                                               _stream_ptr(stream), out.data_ptr()))
         self._keep = (cu_seqlens_dev, workspace)

@@ -1,0 +1,133 @@
+"""Parity at the benchmark's sizes and at full depth.  The oracle costs 0.4-30 TFLOP of fp64 per item, so
+full-size micro-batches are checked on sampled items (an item's output does not depend on its neighbours, which
+the bit-equality tests below establish on the GPU side), and the largest shapes at reduced depth."""
+import numpy as np
+import pytest
+import torch
+
+import eas_synth as S
+from oracle import encoder_oracle as O
+from tests import gpu_util as G
+
+pytestmark = pytest.mark.gpu
+
+
+def _make(cfg, profile="plain"):
+    import paper_2609_31551_b200 as P
+    w = S.make_weights(cfg, profile=profile)
+    return w, P.Encoder(cfg, P.weights_to_device(w))
+
+
+def _out_slices(cfg, items):
+    rows = [S.out_tokens_per_item(cfg, G.item_shape(cfg, it)) for it in items]
+    cu = np.concatenate([[0], np.cumsum(rows)])
+    return [slice(int(a), int(b)) for a, b in zip(cu[:-1], cu[1:])]
+
+
+def test_c1_bench_configuration_sampled_items():
+    """c1 at micro-batch 32, full depth, all SMs: the configuration bench.py times."""
+    cfg = S.get_config("c1")
+    w, enc = _make(cfg)
+    shapes = S.draw_item_shapes(cfg, 32, 3105)
+    items = S.make_items(cfg, shapes, seed=2105)
+    got, out_dev = G.run_gpu(enc, cfg, items)
+    sl = _out_slices(cfg, items)
+    for i in (0, 17, 31):
+        ref = O.encode_item(cfg, w, items[i]).numpy()
+        rel, mabs = G.assert_parity(got[sl[i]], ref, f"c1 mb32 item {i}")
+        print(f"c1 mb32 item {i}: row-rel {rel:.3e} max-abs {mabs:.3e}")
+    # an item encoded alone gives the same bytes as inside the micro-batch, for any SM budget
+    _, alone = G.run_gpu(enc, cfg, [items[17]], sm_budget=37)
+    assert torch.equal(alone, out_dev[sl[17]])
+
+
+def test_c1_full_depth_sharp_profile():
+    cfg = S.get_config("c1")
+    w, enc = _make(cfg, "sharp")
+    items = S.make_items(cfg, [(1, 336, 336)] * 2, seed=2101)
+    ref, _, _ = O.encode_microbatch(cfg, w, items)
+    got, _ = G.run_gpu(enc, cfg, items)
+    print("c1 sharp full depth:", G.assert_parity(got, ref, "c1 sharp"))
+
+
+def test_c2_full_depth_packed_native_resolution():
+    cfg = S.get_config("c2")
+    w, enc = _make(cfg)
+    shapes = [(1, 224, 224), (1, 448, 336), (1, 1344, 224)]       # 256, 768, 1536 tokens
+    items = S.make_items(cfg, shapes, seed=2203)
+    ref, _, _ = O.encode_microbatch(cfg, w, items)
+    got, out_dev = G.run_gpu(enc, cfg, items)
+    print("c2 full depth:", G.assert_parity(got, ref, "c2"))
+    sl = _out_slices(cfg, items)
+    _, alone = G.run_gpu(enc, cfg, [items[1]], sm_budget=74)
+    assert torch.equal(alone, out_dev[sl[1]])
+
+
+def test_c2_largest_image_two_layers():
+    cfg = S.get_config("c2", n_layers=2)
+    w, enc = _make(cfg, "sharp")
+    items = S.make_items(cfg, [(1, 1344, 1344)], seed=2299)       # 9216 tokens
+    ref, _, _ = O.encode_microbatch(cfg, w, items)
+    got, _ = G.run_gpu(enc, cfg, items)
+    print("c2 1344x1344, 2 layers:", G.assert_parity(got, ref, "c2 largest"))
+
+
+def test_c3_full_depth_short_clip_and_long_clip_two_layers():
+    cfg = S.get_config("c3")
+    w, enc = _make(cfg)
+    items = S.make_items(cfg, [(4, 448, 448)], seed=2301)         # 2048 tokens, full depth
+    ref, _, _ = O.encode_microbatch(cfg, w, items)
+    got, _ = G.run_gpu(enc, cfg, items)
+    print("c3 4-frame clip full depth:", G.assert_parity(got, ref, "c3 full depth"))
+    cfg2 = S.get_config("c3", n_layers=2)
+    w2, enc2 = _make(cfg2, "sharp")
+    items2 = S.make_items(cfg2, [(16, 448, 448)], seed=2302)      # 8192 tokens
+    ref2, _, _ = O.encode_microbatch(cfg2, w2, items2)
+    got2, _ = G.run_gpu(enc2, cfg2, items2)
+    print("c3 16-frame clip, 2 layers:", G.assert_parity(got2, ref2, "c3 16 frames"))
+
+
+def test_c3_maximum_clip_is_finite_and_packing_invariant():
+    """64-frame clip = 32768 tokens (the longest sequence of any workload), one layer, GPU-side properties."""
+    cfg = S.get_config("c3", n_layers=1)
+    w, enc = _make(cfg)
+    items = S.make_items(cfg, [(2, 448, 448), (64, 448, 448)], seed=2303)
+    got, out_dev = G.run_gpu(enc, cfg, items)
+    assert np.isfinite(got).all()
+    _, alone = G.run_gpu(enc, cfg, [items[1]], sm_budget=111)
+    assert torch.equal(alone, out_dev[256:])
+    # rows of the short clip against the oracle (it shares the batch with the 32768-token clip)
+    ref = O.encode_item(cfg, w, items[0]).numpy()
+    G.assert_parity(got[:256], ref, "c3 short clip next to the longest")
+
+
+def test_c4_full_depth():
+    cfg = S.get_config("c4")
+    w, enc = _make(cfg)
+    items = S.make_items(cfg, [(3000, 128, 1), (1000, 128, 1)], seed=2401)
+    ref, _, _ = O.encode_microbatch(cfg, w, items)
+    got, out_dev = G.run_gpu(enc, cfg, items)
+    print("c4 full depth:", G.assert_parity(got, ref, "c4"))
+    for budget in (37, 74, 111):
+        _, b = G.run_gpu(enc, cfg, items, sm_budget=budget)
+        assert torch.equal(b, out_dev), budget
+
+
+def test_degenerate_micro_batches():
+    """One item; the smallest legal items; many tiny items (64) in one micro-batch."""
+    cfg = S.get_config("c2", n_layers=2)
+    w, enc = _make(cfg)
+    tiny = S.make_items(cfg, [(1, 28, 28)], seed=1)               # 4 tokens -> 1 output row
+    ref, _, _ = O.encode_microbatch(cfg, w, tiny)
+    got, _ = G.run_gpu(enc, cfg, tiny)
+    G.assert_parity(got, ref, "single 2x2-patch image")
+    many = S.make_items(cfg, [(1, 28, 28 * (1 + i % 3)) for i in range(64)], seed=2)
+    ref, _, _ = O.encode_microbatch(cfg, w, many)
+    got, _ = G.run_gpu(enc, cfg, many)
+    G.assert_parity(got, ref, "64 tiny images")
+    cfg4 = S.get_config("c4", n_layers=1)
+    w4, enc4 = _make(cfg4)
+    a = S.make_items(cfg4, [(2, 128, 1)] * 3, seed=3)             # 1 token per clip
+    ref, _, _ = O.encode_microbatch(cfg4, w4, a)
+    got, _ = G.run_gpu(enc4, cfg4, a)
+    G.assert_parity(got, ref, "one-token audio clips")
