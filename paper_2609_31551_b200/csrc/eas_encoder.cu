@@ -86,6 +86,21 @@ static eas_status make_a_tmap(CUtensorMap* m, const void* a, int64_t run, int64_
   return make_tmap(m, a, 3, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B);
 }
 
+// output [rows, ld] as a store / reduce target: 32-row boxes whose rows are 128 bytes (64 bf16 or 32 fp32)
+static eas_status make_out_tmap(CUtensorMap* m, const void* out, bool fp32, int64_t cols, int64_t ld, int64_t rows) {
+  PFN_cuTensorMapEncodeTiled_v12000 fn = get_encode_fn();
+  if (fn == nullptr) return fail(EAS_ERR_CUDA, "cuTensorMapEncodeTiled is not available from the driver");
+  const cuuint64_t gdim[2] = {static_cast<cuuint64_t>(cols), static_cast<cuuint64_t>(rows)};
+  const cuuint64_t gstr[1] = {static_cast<cuuint64_t>(ld) * (fp32 ? 4 : 2)};
+  const cuuint32_t box[2] = {fp32 ? 32u : 64u, 32u};
+  const cuuint32_t es[2] = {1, 1};
+  CUresult r = fn(m, fp32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(out),
+                  gdim, gstr, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                  CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return fail(EAS_ERR_CUDA, "cuTensorMapEncodeTiled (output) failed with code %d", static_cast<int>(r));
+  return EAS_OK;
+}
+
 // ------------------------------------------------------------------------------------ handle
 struct Linear {
   const bf16* w = nullptr;   // [N, K] (possibly re-laid)
@@ -484,6 +499,12 @@ static eas_status launch_gemm(const GemmCall& g, int budget, cudaStream_t stream
   p.row_map = g.row_map; p.pos_idx = g.pos_idx; p.pos = g.pos;
   p.rope_cs = g.rope_cs; p.rope_pairs = g.rope_pairs; p.rope_ncols = g.rope_ncols; p.head_dim = g.head_dim > 0 ? g.head_dim : 64;
   p.status = status;
+  // TMA-store epilogue whenever output rows are the A rows and any residual is accumulated in place
+  p.use_tma_out = (g.row_map == nullptr && g.pos == nullptr && (g.resid == nullptr || g.resid == g.out)) ? 1 : 0;
+  if (p.use_tma_out) {
+    const int64_t out_cols = g.act == ACT_SWIGLU ? L.N / 2 : L.N;
+    EAS_TRY(make_out_tmap(&p.tma_out, g.out, g.out_fp32 != 0, out_cols, g.ldo, g.M));
+  }
   const int tiles = p.m_blocks * p.n_blocks;
   const int grid = std::min(budget, tiles);
   void (*kern)(GemmParams) = nullptr;

@@ -3,7 +3,8 @@
 //   warp 0      TMA producer: 128x64 A tiles and 256x64 W tiles into a 4-stage shared-memory ring
 //   warp 1      UMMA issuer: tcgen05.mma 128x256x16, fp32 accumulators in TMEM, two accumulator
 //               buffers (2 x 256 columns) so that the epilogue of tile i overlaps the main loop of tile i+1
-//   warps 2..9  epilogue: tcgen05.ld -> bias / activation / rotary / residual -> global stores
+//   warps 2..9  epilogue: tcgen05.ld -> bias / activation / rotary -> swizzled shared-memory staging -> TMA store
+//               (TMA reduce-add into the fp32 residual stream); scatter epilogues (row maps) store directly
 //
 // The grid is `sm_budget` CTAs (one per SM: the shared-memory request excludes a second resident
 // CTA) and each CTA walks tiles  blockIdx.x, blockIdx.x + gridDim.x, ...  in a fixed order, so the
@@ -20,7 +21,11 @@ constexpr int kGemmThreads = 64 + 32 * kEpiWarps;
 constexpr int kABytes = kBM * kBK * 2;            // 16 KB
 constexpr int kBBytes = kBN * kBK * 2;            // 32 KB
 constexpr int kStageBytes = kABytes + kBBytes;    // 48 KB
-constexpr int kGemmSmemBytes = kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
+constexpr int kStagingOff = kStages * kStageBytes;             // 8 epilogue warps x 4 KB output staging (TMA store source)
+constexpr int kBiasOff = kStagingOff + kEpiWarps * 4096;       // 2 x 256 fp32 bias values of the current tiles
+constexpr int kBarOff = kBiasOff + 2 * 256 * 4;
+constexpr int kGemmSmemBytes = kBarOff + 128 /*barriers*/ + 896 /*alignment slack: the base is 128-byte aligned at least*/;
+static_assert(kGemmSmemBytes <= 232448, "exceeds the 227 KB shared memory of an SM");
 constexpr int kTmemCols = 512;
 constexpr int kPanelM = 8;                        // m-blocks per rasterisation panel (L2 reuse of W tiles)
 
@@ -30,6 +35,8 @@ enum { OUT_BF16 = 0, OUT_F32 = 1 };
 struct alignas(64) GemmParams {
   CUtensorMap tma_a;      // 3-D: {K-run, phase, rows}; box {64, 1, 128}
   CUtensorMap tma_b;      // 2-D: {K, N}; box {64, 256}
+  CUtensorMap tma_out;    // 2-D over out: box {64 bf16 | 32 fp32, 32 rows}, 128-byte swizzle (valid if use_tma_out)
+  int use_tma_out;        // 1: epilogue stages 32-row sub-tiles in shared memory and stores them with TMA
   int M, N;               // rows of A walked by tiles; rows of W
   int k_blocks;           // K / 64 (K padded with zeros by the caller or by TMA fill)
   int kb_per_tap;         // k-blocks per convolution tap (== k_blocks for a plain GEMM)
@@ -60,15 +67,16 @@ __device__ __forceinline__ void tile_coords(int tile, int m_blocks, int n_blocks
 
 template <int ACT, int OUT>
 __global__ void __launch_bounds__(kGemmThreads, 1) gemm_kernel(const __grid_constant__ GemmParams p) {
-  extern __shared__ uint8_t smem_raw[];
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
   // 1024-byte alignment: the 128-byte swizzle pattern repeats every 8 rows of 128 bytes
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kStages * kStageBytes);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kBarOff);
   uint64_t* full_bar = bars;                    // [kStages]  TMA -> MMA
   uint64_t* empty_bar = bars + kStages;         // [kStages]  MMA -> TMA
   uint64_t* acc_full = bars + 2 * kStages;      // [2]        MMA -> epilogue
   uint64_t* acc_empty = bars + 2 * kStages + 2; // [2]        epilogue -> MMA
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kStages + 4);
+  uint64_t* bias_bar = bars + 2 * kStages + 4;  // [2]        epilogue warps: bias values staged
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kStages + 6);
   volatile uint32_t* abort_flag = tmem_slot + 1;
 
   const int warp = threadIdx.x >> 5;
@@ -77,11 +85,12 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_kernel(const __grid_cons
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
-    for (int a = 0; a < 2; ++a) { mbar_init(&acc_full[a], 1); mbar_init(&acc_empty[a], kEpiWarps); }
+    for (int a = 0; a < 2; ++a) { mbar_init(&acc_full[a], 1); mbar_init(&acc_empty[a], kEpiWarps); mbar_init(&bias_bar[a], kEpiWarps); }
     *abort_flag = 0;
     mbar_fence_init();
     tma_prefetch_desc(&p.tma_a);
     tma_prefetch_desc(&p.tma_b);
+    if (p.use_tma_out) tma_prefetch_desc(&p.tma_out);
   }
   if (warp == 1) {
     tmem_alloc(tmem_slot, kTmemCols);
@@ -164,6 +173,130 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_kernel(const __grid_cons
       tile_coords(tile, p.m_blocks, p.n_blocks, mb, nb);
       const uint32_t acc = tcount & 1u;
       const uint32_t acc_ph = (tcount >> 1) & 1u;
+      if (p.use_tma_out) {
+        // ---- staged path: bias from shared memory, 32-row sub-tiles written to a swizzled staging buffer
+        //      and stored (or reduce-added, for the fp32 residual stream) by TMA; rows >= M are clipped by TMA
+        float* sbias = reinterpret_cast<float*>(smem + kBiasOff) + acc * 256;
+        {
+          const int col = nb * kBN + ew * 32 + lane;
+          sbias[ew * 32 + lane] = col < p.N ? __bfloat162float(p.bias[col]) : 0.f;
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&bias_bar[acc]);
+        }
+        if (!mbar_wait(&acc_full[acc], acc_ph, abort_flag)) { ok = false; break; }
+        if (!mbar_wait(&bias_bar[acc], acc_ph, abort_flag)) { ok = false; break; }
+        tc_fence_after_sync();
+        uint8_t* stage = smem + kStagingOff + ew * 4096;
+        uint8_t* srow = stage + lane * 128;
+        const int sw = lane & 7;
+        const int arow = mb * kBM + quarter * 32 + lane;
+        const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + acc * kBN + half * 128;
+        const int ycoord = mb * kBM + quarter * 32;
+
+        auto finish_chunk = [&](float (&v)[32], int c) {   // bias, rotary, activation on 32 accumulator columns
+          const int col0 = nb * kBN + half * 128 + c * 32;
+          const float4* b4 = reinterpret_cast<const float4*>(sbias + half * 128 + c * 32);
+#pragma unroll
+          for (int q = 0; q < 8; ++q) {
+            const float4 b = b4[q];
+            v[4 * q] += b.x; v[4 * q + 1] += b.y; v[4 * q + 2] += b.z; v[4 * q + 3] += b.w;
+          }
+          if (p.rope_cs != nullptr && col0 < p.rope_ncols && arow < p.M) {
+            const float2* cs = p.rope_cs + static_cast<long long>(arow) * p.rope_pairs;
+            int pi = (col0 % p.head_dim) >> 1;
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+              const float2 t = __ldg(cs + pi);
+              const float x0 = v[2 * j], x1 = v[2 * j + 1];
+              v[2 * j] = x0 * t.x - x1 * t.y;
+              v[2 * j + 1] = x1 * t.x + x0 * t.y;
+              if (++pi == p.rope_pairs) pi = 0;
+            }
+          }
+          if (ACT == ACT_GELU) {
+#pragma unroll
+            for (int i = 0; i < 32; ++i) v[i] = gelu_erf(v[i]);
+          }
+        };
+        auto staging_free = [&]() {       // the previous bulk store has finished READING the staging buffer
+          if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+          __syncwarp();
+        };
+        auto store_subtile = [&](int x) { // one TMA store / reduce-add of the 32-row staging buffer at column x
+          fence_proxy_async_smem();
+          __syncwarp();
+          if (lane == 0) {
+            if (OUT == OUT_F32 && p.resid != nullptr) {
+              asm volatile("cp.reduce.async.bulk.tensor.2d.global.shared::cta.add.bulk_group [%0, {%2, %3}], [%1];"
+                           ::"l"(reinterpret_cast<uint64_t>(&p.tma_out)), "r"(smem_u32(stage)), "r"(x), "r"(ycoord) : "memory");
+            } else {
+              asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
+                           ::"l"(reinterpret_cast<uint64_t>(&p.tma_out)), "r"(smem_u32(stage)), "r"(x), "r"(ycoord) : "memory");
+            }
+            asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+          }
+        };
+
+#pragma unroll 1
+        for (int pr = 0; pr < 2; ++pr) {            // two chunks (64 accumulator columns) per round
+          uint32_t r0[32], r1[32];
+          __syncwarp();
+          tmem_ld_32x32(taddr + pr * 64, r0);
+          tmem_ld_32x32(taddr + pr * 64 + 32, r1);
+          tmem_ld_wait();
+          float v0[32], v1[32];
+#pragma unroll
+          for (int i = 0; i < 32; ++i) { v0[i] = __uint_as_float(r0[i]); v1[i] = __uint_as_float(r1[i]); }
+          finish_chunk(v0, pr * 2);
+          finish_chunk(v1, pr * 2 + 1);
+          const int col0 = nb * kBN + half * 128 + pr * 64;
+          if (OUT == OUT_F32) {
+            // 32 fp32 columns = one 128-byte staging row; two sub-tiles per round
+#pragma unroll
+            for (int h2 = 0; h2 < 2; ++h2) {
+              float (&v)[32] = h2 ? v1 : v0;
+              staging_free();
+#pragma unroll
+              for (int q = 0; q < 8; ++q)
+                *reinterpret_cast<float4*>(srow + ((q ^ sw) << 4)) = make_float4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
+              if (col0 + h2 * 32 < p.N) store_subtile(col0 + h2 * 32);
+            }
+          } else if (ACT == ACT_SWIGLU) {
+            // (gate, up) pairs -> 32 outputs per round; the 64 outputs of both rounds form one staging row
+            if (pr == 0) staging_free();
+#pragma unroll
+            for (int h2 = 0; h2 < 2; ++h2) {
+              float (&v)[32] = h2 ? v1 : v0;
+              uint32_t w[8];
+#pragma unroll
+              for (int j = 0; j < 8; ++j)
+                w[j] = pack_bf16x2(silu_f(v[4 * j]) * v[4 * j + 1], silu_f(v[4 * j + 2]) * v[4 * j + 3]);
+              const int q0 = pr * 4 + h2 * 2;
+              *reinterpret_cast<uint4*>(srow + (((q0) ^ sw) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
+              *reinterpret_cast<uint4*>(srow + (((q0 + 1) ^ sw) << 4)) = make_uint4(w[4], w[5], w[6], w[7]);
+            }
+            if (pr == 1 && nb * kBN + half * 128 < p.N) store_subtile((nb * kBN + half * 128) >> 1);
+          } else {
+            // 64 bf16 columns = one 128-byte staging row
+            staging_free();
+#pragma unroll
+            for (int h2 = 0; h2 < 2; ++h2) {
+              float (&v)[32] = h2 ? v1 : v0;
+#pragma unroll
+              for (int q = 0; q < 4; ++q)
+                *reinterpret_cast<uint4*>(srow + (((h2 * 4 + q) ^ sw) << 4)) =
+                    make_uint4(pack_bf16x2(v[8 * q], v[8 * q + 1]), pack_bf16x2(v[8 * q + 2], v[8 * q + 3]),
+                               pack_bf16x2(v[8 * q + 4], v[8 * q + 5]), pack_bf16x2(v[8 * q + 6], v[8 * q + 7]));
+            }
+            if (col0 < p.N) store_subtile(col0);
+          }
+        }
+        tc_fence_before_sync();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&acc_empty[acc]);
+        continue;
+      }
+
       if (!mbar_wait(&acc_full[acc], acc_ph, abort_flag)) { ok = false; break; }
       tc_fence_after_sync();
 
@@ -276,6 +409,8 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_kernel(const __grid_cons
       __syncwarp();
       if (lane == 0) mbar_arrive(&acc_empty[acc]);
     }
+    // bulk stores still reading the staging buffer must finish before the CTA's shared memory is released
+    if (p.use_tma_out && lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
   }
 
   tc_fence_before_sync();

@@ -45,6 +45,22 @@ def test_gemm_epilogues(M, N, K, act, out_fp32):
     assert not bad.any(), f"{int(bad.sum())} of {bad.numel()} wrong, max err {(got - y).abs().max():.4e}, first bad {bad.nonzero()[:5].tolist()}"
 
 
+@pytest.mark.parametrize("M,N,K", [(300, 512, 128), (1000, 1024, 1024), (77, 288, 192)])
+def test_gemm_residual_accumulated_in_place(M, N, K):
+    """fp32 residual stream updated in place (x += A W^T + b): the path the encoder's proj / fc2 GEMMs take."""
+    import paper_2609_31551_b200 as P
+    rng = np.random.Generator(np.random.PCG64(M + N))
+    A, W, b = _bf16_exact(rng, (M, K)), _bf16_exact(rng, (N, K), 0.05), _bf16_exact(rng, (N,), 0.5)
+    r = rng.standard_normal((M, N)).astype(np.float32)
+    y = O.linear(O._t(A), O._t(W), O._t(b)) + O._t(r)
+    x = torch.from_numpy(r).cuda()
+    out, status = P.kernel_gemm(_dev(A), _dev(W), _dev(b), act=0, out_fp32=True, resid=x, out=x)
+    torch.cuda.synchronize()
+    assert int(status[0]) == 0
+    err = (x.double().cpu() - y).abs()
+    assert err.max() <= 1e-5 * float(y.abs().max()) + 2e-3 * max(1.0, float(K) ** 0.5 * 0.05), err.max()
+
+
 def test_gemm_is_independent_of_sm_budget():
     import paper_2609_31551_b200 as P
     rng = np.random.Generator(np.random.PCG64(5))
