@@ -6,8 +6,9 @@
 //
 //   warp 0       TMA producer: Q tiles (double buffered across units), K/V tiles through a ring
 //   warp 1       UMMA issuer:  S = Q K^T (128x128x{64|80}) into TMEM, O += P V (128x{64|80}x128) in TMEM
-//   warps 2..5   softmax warpgroup of tile A: one thread per query row
-//   warps 6..9   softmax warpgroup of tile B
+//   warps 2, 3   idle (they complete the first warpgroup, whose registers are handed to the softmax warps)
+//   warps 4..7   softmax warpgroup of tile A: one thread per query row
+//   warps 8..11  softmax warpgroup of tile B
 //
 // A softmax thread reads its row of S from TMEM, keeps a running reference maximum m and sum l, writes
 // P = exp2((s - m) * scale) as bf16 into shared memory (K-major, 128-byte swizzle: the A operand of P V).
@@ -19,7 +20,7 @@
 
 namespace eas {
 
-constexpr int kTcThreads = 320;
+constexpr int kTcThreads = 384;
 constexpr int kTcTile = 128;            // query rows per tile and keys per K/V tile
 constexpr float kRescaleThreshold = 8.0f;
 
@@ -69,6 +70,54 @@ __device__ __forceinline__ void tmem_st_32x16(uint32_t taddr, const uint32_t (&r
       : "memory");
 }
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+template <int OFF>
+__device__ __forceinline__ void tmem_ld_32x32_at(uint32_t taddr, uint32_t (&r)[128]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[OFF + 0]), "=r"(r[OFF + 1]), "=r"(r[OFF + 2]), "=r"(r[OFF + 3]), "=r"(r[OFF + 4]), "=r"(r[OFF + 5]),
+        "=r"(r[OFF + 6]), "=r"(r[OFF + 7]), "=r"(r[OFF + 8]), "=r"(r[OFF + 9]), "=r"(r[OFF + 10]), "=r"(r[OFF + 11]),
+        "=r"(r[OFF + 12]), "=r"(r[OFF + 13]), "=r"(r[OFF + 14]), "=r"(r[OFF + 15]), "=r"(r[OFF + 16]), "=r"(r[OFF + 17]),
+        "=r"(r[OFF + 18]), "=r"(r[OFF + 19]), "=r"(r[OFF + 20]), "=r"(r[OFF + 21]), "=r"(r[OFF + 22]), "=r"(r[OFF + 23]),
+        "=r"(r[OFF + 24]), "=r"(r[OFF + 25]), "=r"(r[OFF + 26]), "=r"(r[OFF + 27]), "=r"(r[OFF + 28]), "=r"(r[OFF + 29]),
+        "=r"(r[OFF + 30]), "=r"(r[OFF + 31])
+      : "r"(taddr + OFF)
+      : "memory");
+}
+// packed fp32x2 arithmetic (two lanes per instruction on the FMA pipe)
+__device__ __forceinline__ uint64_t pack2(float lo, float hi) {
+  uint64_t d;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(d) : "f"(lo), "f"(hi));
+  return d;
+}
+__device__ __forceinline__ void unpack2(uint64_t v, float& lo, float& hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t ffma2(uint64_t a, uint64_t b, uint64_t c) {
+  uint64_t d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ uint64_t fadd2(uint64_t a, uint64_t b) {
+  uint64_t d;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+__device__ __forceinline__ float fmax3(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
+// Register re-balancing between warpgroups.  The pool is the CTA's launch allocation (168 x 384 registers): the
+// sum over warpgroups of 128 x their limit must stay BELOW it, or setmaxnreg.inc waits forever.
+constexpr int kRegsLight = 112, kRegsSoftmax = 192;
+static_assert(128 * kRegsLight + 256 * kRegsSoftmax < 168 * 384, "setmaxnreg budget exceeds the CTA's register allocation");
+template <int N>
+__device__ __forceinline__ void setmaxnreg_inc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N)); }
+template <int N>
+__device__ __forceinline__ void setmaxnreg_dec() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N)); }
 
 struct UnitInfo {
   int head, q0, S, n_kv, n_q;
@@ -141,6 +190,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_tc_kernel(const __grid_con
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
+    setmaxnreg_dec<kRegsLight>();
     if (lane == 0) {
       uint32_t kv_it = 0, u_cnt = 0;
       bool ok = true;
@@ -174,6 +224,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_tc_kernel(const __grid_con
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ UMMA issuer
+    setmaxnreg_dec<kRegsLight>();
     if (lane == 0) {
       constexpr uint32_t idesc_s = make_idesc_bf16(128, 128, 0, 0);     // S = Q K^T, both K-major
       constexpr uint32_t idesc_o_lo = make_idesc_bf16(128, 64, 0, 1);   // O[:, 0:64] += P V, V is MN-major
@@ -248,9 +299,12 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_tc_kernel(const __grid_con
         if (ok) umma_commit(&q_empty[qb]);
       }
     }
+  } else if (warp < 4) {
+    setmaxnreg_dec<kRegsLight>();
   } else {
     // ------------------------------------------------------------------ softmax warpgroups
-    const int w = (warp - 2) >> 2;                 // 0: tile A, 1: tile B
+    setmaxnreg_inc<kRegsSoftmax>();
+    const int w = (warp - 4) >> 2;                 // 0: tile A, 1: tile B
     const int quarter = warp & 3;                  // TMEM lane quarter of this warp
     const int row = quarter * 32 + lane;           // query row inside the tile == TMEM lane
     const uint32_t lane_addr = static_cast<uint32_t>(quarter * 32) << 16;
@@ -269,22 +323,25 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_tc_kernel(const __grid_con
         if (!mbar_wait(&s_full[w], n & 1u, abort_flag)) { ok = false; break; }
         tc_fence_after_sync();
         const int valid = min(kTcTile, u.S - j * kTcTile);     // keys of this tile that belong to the item
-        // pass 1: row maximum
-        float mx = -INFINITY;
-#pragma unroll 1
-        for (int c = 0; c < 4; ++c) {
-          uint32_t raw[32];
-          __syncwarp();
-          tmem_ld_32x32(s_addr + c * 32, raw);
-          tmem_ld_wait();
-          if (valid >= (c + 1) * 32) {
+        // the whole score row (128 fp32) in registers: four loads, one wait
+        uint32_t sr[128];
+        __syncwarp();
+        tmem_ld_32x32_at<0>(s_addr, sr);
+        tmem_ld_32x32_at<32>(s_addr, sr);
+        tmem_ld_32x32_at<64>(s_addr, sr);
+        tmem_ld_32x32_at<96>(s_addr, sr);
+        tmem_ld_wait();
+        if (valid < kTcTile) {                                  // last tile of the item: keys past its end
 #pragma unroll
-            for (int i = 0; i < 32; ++i) mx = fmaxf(mx, __uint_as_float(raw[i]));
-          } else {
-#pragma unroll
-            for (int i = 0; i < 32; ++i) if (c * 32 + i < valid) mx = fmaxf(mx, __uint_as_float(raw[i]));
-          }
+          for (int i = 0; i < 128; ++i) if (i >= valid) sr[i] = 0xff800000u;   // -inf
         }
+        float mx0 = -INFINITY, mx1 = -INFINITY;
+#pragma unroll
+        for (int i = 0; i < 128; i += 4) {
+          mx0 = fmax3(mx0, __uint_as_float(sr[i]), __uint_as_float(sr[i + 1]));
+          mx1 = fmax3(mx1, __uint_as_float(sr[i + 2]), __uint_as_float(sr[i + 3]));
+        }
+        const float mx = fmaxf(mx0, mx1);
         // reference maximum: moves only when the row maximum grew by more than the threshold
         float corr = 1.0f;
         bool rescale = false;
@@ -297,25 +354,33 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_tc_kernel(const __grid_con
         }
         l *= corr;
         const float mb = m_used * p.scale_log2;
-        // pass 2: probabilities, kept packed in registers until the P buffer is free
+        const uint64_t scale2 = pack2(p.scale_log2, p.scale_log2);
+        const uint64_t nmb2 = pack2(-mb, -mb);
+        // probabilities, kept packed in registers until the P buffer is free
         uint32_t pk[64];
+        uint64_t acc0 = 0, acc1 = 0, acc2 = 0, acc3 = 0;       // (0.f, 0.f) pairs
 #pragma unroll
-        for (int c = 0; c < 4; ++c) {
-          uint32_t raw[32];
-          __syncwarp();
-          tmem_ld_32x32(s_addr + c * 32, raw);
-          tmem_ld_wait();
-          float sum = 0.f;
+        for (int i = 0; i < 64; i += 4) {
 #pragma unroll
-          for (int i = 0; i < 32; i += 2) {
-            float p0 = fast_ex2(fmaf(__uint_as_float(raw[i]), p.scale_log2, -mb));
-            float p1 = fast_ex2(fmaf(__uint_as_float(raw[i + 1]), p.scale_log2, -mb));
-            if (c * 32 + i >= valid) p0 = 0.f;
-            if (c * 32 + i + 1 >= valid) p1 = 0.f;
-            sum += p0 + p1;
-            pk[c * 16 + (i >> 1)] = pack_bf16x2(p0, p1);
+          for (int q = 0; q < 4; ++q) {
+            const uint64_t t = ffma2(pack2(__uint_as_float(sr[2 * (i + q)]), __uint_as_float(sr[2 * (i + q) + 1])), scale2, nmb2);
+            float t0, t1;
+            unpack2(t, t0, t1);
+            const float p0 = fast_ex2(t0);
+            const float p1 = fast_ex2(t1);
+            const uint64_t pp = pack2(p0, p1);
+            if (q == 0) acc0 = fadd2(acc0, pp);
+            if (q == 1) acc1 = fadd2(acc1, pp);
+            if (q == 2) acc2 = fadd2(acc2, pp);
+            if (q == 3) acc3 = fadd2(acc3, pp);
+            pk[i + q] = pack_bf16x2(p0, p1);
           }
-          l += sum;
+        }
+        {
+          const uint64_t a = fadd2(fadd2(acc0, acc1), fadd2(acc2, acc3));
+          float a0, a1;
+          unpack2(a, a0, a1);
+          l += a0 + a1;
         }
         // S has been read: the issuer may overwrite it with the next tile's scores once p_ready fires.
         // The previous P V must be complete before P is overwritten or O is touched.
