@@ -135,6 +135,27 @@ int64_t eas_encoder_out_rows(const eas_encoder* enc, const int32_t* cu_seqlens_h
 eas_status eas_encode_microbatch(eas_encoder* enc, const eas_packed_inputs* in, const int32_t* cu_seqlens,
                                  int32_t sm_budget, void* stream, void* out_embeddings);
 
+/* The paper has no counterpart for this entry point; it exists for callers that cannot allocate device memory.
+ * An encode worker that shares its GPU with a prefill worker (Section 3.4 co-locates them) typically starts after
+ * the neighbour has claimed the rest of HBM for its KV cache, and runs inside a serving loop where an allocation may
+ * fail, or may make the whole device wait while the driver grows its heap.  Such a caller can use this variant of
+ * eas_encode_microbatch: same arguments, same result, but the scratch the forward pass needs comes from an array of
+ * EAS_STATIC_WORKSPACE_BYTES that is part of the library image, so the call itself allocates nothing (no cudaMalloc,
+ * cudaFree, or allocating library routine).  in->workspace and in->workspace_bytes are ignored; the caller still
+ * provides data, cu_seqlens and out_embeddings.
+ *  - Limit: the micro-batch must fit the built-in scratch (about 20 KB per token for a d=256 model, 90 KB per token
+ *    for d=1280); a larger one is rejected with EAS_ERR_WORKSPACE and a message that states both sizes.
+ *  - Cost: every GPU on which this library is loaded holds the array until the process exits.
+ *  - The first call on each device looks up the array's device address (cudaGetSymbolAddress, with that device
+ *    current).  Make that first call before starting any stream capture.
+ *  - All calls on one device share the one array, which keeps whatever the previous call left in it.  The forward
+ *    pass clears its status word itself and writes every other scratch region before reading it, so nothing has to
+ *    be zeroed by the caller; but two calls whose kernels overlap on the GPU (different streams, or different
+ *    handles) would race on it.  Serialise them, or use eas_encode_microbatch with separate workspaces. */
+#define EAS_STATIC_WORKSPACE_BYTES (32u << 20)
+eas_status eas_encode_microbatch_static(eas_encoder* enc, const eas_packed_inputs* in, const int32_t* cu_seqlens,
+                                        int32_t sm_budget, void* stream, void* out_embeddings);
+
 /* Synchronises `stream`, then reads and clears the device status word of the last call's workspace:
  * EAS_OK, EAS_ERR_DEVICE_TIMEOUT, EAS_ERR_DEVICE_CHECK or EAS_ERR_CUDA. */
 eas_status eas_encoder_status(eas_encoder* enc, void* stream);

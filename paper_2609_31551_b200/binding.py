@@ -15,7 +15,7 @@ STATUS_NAMES = {0: "EAS_OK", 1: "EAS_ERR_INVALID_ARG", 2: "EAS_ERR_UNSUPPORTED",
 
 EXPORTED_SYMBOLS = [
     "eas_encoder_create", "eas_encoder_weight_arena_bytes", "eas_encoder_workspace_bytes", "eas_encoder_out_rows",
-    "eas_encode_microbatch", "eas_encoder_status", "eas_encoder_last_launch_count", "eas_encoder_set_attention_impl",
+    "eas_encode_microbatch", "eas_encode_microbatch_static", "eas_encoder_status", "eas_encoder_last_launch_count", "eas_encoder_set_attention_impl",
     "eas_encoder_enable_timing", "eas_encoder_timing_read", "eas_last_error", "eas_encoder_destroy", "eas_kernel_gemm", "eas_kernel_norm", "eas_kernel_attention",
 ]
 
@@ -69,6 +69,8 @@ def load_library():
     lib.eas_encoder_out_rows.argtypes = [C.c_void_p, C.POINTER(C.c_int32), C.c_int32]
     lib.eas_encode_microbatch.restype = C.c_int
     lib.eas_encode_microbatch.argtypes = [C.c_void_p, C.POINTER(PackedInputs), C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p]
+    lib.eas_encode_microbatch_static.restype = C.c_int
+    lib.eas_encode_microbatch_static.argtypes = [C.c_void_p, C.POINTER(PackedInputs), C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p]
     lib.eas_encoder_status.restype = C.c_int
     lib.eas_encoder_status.argtypes = [C.c_void_p, C.c_void_p]
     lib.eas_encoder_last_launch_count.restype = C.c_int32
@@ -214,6 +216,20 @@ class Encoder:
         _check(self.lib.eas_encode_microbatch(self.handle, C.byref(pin), cu_seqlens_dev.data_ptr(), sm_budget,
                                               _stream_ptr(stream), out.data_ptr()))
         self._keep = (cu_seqlens_dev, workspace)
+        return out
+
+    def encode_microbatch_static(self, data: torch.Tensor, item_shapes, item_offsets, cu_seqlens_host,
+                                 cu_seqlens_dev: torch.Tensor, out: torch.Tensor, sm_budget: int = 0, stream=None):
+        """eas_encode_microbatch_static: the forward pass on the scratch built into the library.  Nothing is
+        allocated here either: the caller passes the device cu_seqlens and the output tensor."""
+        n = len(item_shapes)
+        shp = np.ascontiguousarray(item_shapes, dtype=np.int32).reshape(n, 3)
+        offs = np.ascontiguousarray(item_offsets, dtype=np.int64)
+        cu = np.ascontiguousarray(cu_seqlens_host, dtype=np.int32)
+        pin = PackedInputs(data.data_ptr(), n, shp.ctypes.data_as(C.POINTER(C.c_int32)),
+                           offs.ctypes.data_as(C.POINTER(C.c_int64)), cu.ctypes.data_as(C.POINTER(C.c_int32)), None, 0)
+        _check(self.lib.eas_encode_microbatch_static(self.handle, C.byref(pin), cu_seqlens_dev.data_ptr(), sm_budget,
+                                                     _stream_ptr(stream), out.data_ptr()))
         return out
 
     def status(self, stream=None):

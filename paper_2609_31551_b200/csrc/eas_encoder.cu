@@ -13,6 +13,7 @@
 #include <cstring>
 #include <map>
 #include <memory>
+#include <mutex>
 #include <string>
 #include <vector>
 
@@ -634,16 +635,18 @@ static eas_status launch_attention(const bf16* qkv, bf16* out, const int32_t* cu
 }
 
 // ------------------------------------------------------------------------------------ the forward pass
-extern "C" eas_status eas_encode_microbatch(eas_encoder* e, const eas_packed_inputs* in, const int32_t* cu_dev,
-                                            int32_t sm_budget, void* stream_v, void* out_embeddings) {
+// The forward pass.  `workspace` / `workspace_bytes` override the fields of `in` (the entry points differ only in
+// where the scratch comes from).
+static eas_status encode_impl(eas_encoder* e, const eas_packed_inputs* in, void* workspace, size_t workspace_bytes,
+                              const int32_t* cu_dev, int32_t sm_budget, void* stream_v, void* out_embeddings) {
   if (e == nullptr || in == nullptr) return fail(EAS_ERR_INVALID_ARG, "encoder or inputs are null");
   if (in->data == nullptr || in->item_shape == nullptr || in->item_offset == nullptr || in->cu_seqlens_host == nullptr ||
-      in->workspace == nullptr || cu_dev == nullptr || out_embeddings == nullptr)
+      workspace == nullptr || cu_dev == nullptr || out_embeddings == nullptr)
     return fail(EAS_ERR_INVALID_ARG, "a required pointer is null");
   const int n = in->n_items;
   if (n < 1 || n > EAS_MAX_ITEMS) return fail(EAS_ERR_INVALID_ARG, "n_items %d outside 1..%d", n, static_cast<int>(EAS_MAX_ITEMS));
   if (sm_budget < 0 || sm_budget > e->sm_count) return fail(EAS_ERR_INVALID_ARG, "sm_budget %d outside 0..%d", sm_budget, e->sm_count);
-  if ((reinterpret_cast<uintptr_t>(in->workspace) & 1023) != 0) return fail(EAS_ERR_INVALID_ARG, "workspace is not 1024-byte aligned");
+  if ((reinterpret_cast<uintptr_t>(workspace) & 1023) != 0) return fail(EAS_ERR_INVALID_ARG, "workspace is not 1024-byte aligned");
   if ((reinterpret_cast<uintptr_t>(in->data) & 15) != 0 || (reinterpret_cast<uintptr_t>(out_embeddings) & 15) != 0)
     return fail(EAS_ERR_INVALID_ARG, "data / out_embeddings must be 16-byte aligned");
   const int budget = sm_budget == 0 ? e->sm_count : sm_budget;
@@ -688,10 +691,10 @@ extern "C" eas_status eas_encode_microbatch(eas_encoder* e, const eas_packed_inp
   items.aux_start[n] = aux;
   const int64_t T = cu[n];
   const Plan pl = make_plan(e, T, n);
-  if (in->workspace_bytes < pl.total) return fail(EAS_ERR_WORKSPACE, "workspace too small: %zu bytes given, %zu needed", in->workspace_bytes, pl.total);
+  if (workspace_bytes < pl.total) return fail(EAS_ERR_WORKSPACE, "workspace too small: %zu bytes available, %zu needed", workspace_bytes, pl.total);
 
   cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
-  uint8_t* ws = static_cast<uint8_t*>(in->workspace);
+  uint8_t* ws = static_cast<uint8_t*>(workspace);
   uint32_t* status = reinterpret_cast<uint32_t*>(ws + pl.status);
   float* x = reinterpret_cast<float*>(ws + pl.x);
   bf16* nbuf = reinterpret_cast<bf16*>(ws + pl.n);
@@ -865,6 +868,57 @@ extern "C" eas_status eas_encode_microbatch(eas_encoder* e, const eas_packed_inp
   EAS_TRY(mark(e, -1, stream));
   e->last_launches = launches;
   return EAS_OK;
+}
+
+extern "C" eas_status eas_encode_microbatch(eas_encoder* e, const eas_packed_inputs* in, const int32_t* cu_dev,
+                                            int32_t sm_budget, void* stream_v, void* out_embeddings) {
+  if (in == nullptr) return fail(EAS_ERR_INVALID_ARG, "encoder or inputs are null");
+  return encode_impl(e, in, in->workspace, in->workspace_bytes, cu_dev, sm_budget, stream_v, out_embeddings);
+}
+
+// ------------------------------------------------------------------------------------ scratch baked into the library
+// Scratch for callers that must not allocate: it lives in the library image, so every GPU that loads the
+// library carries it until the process exits.  In host code the array's name is only a host-side stand-in, never
+// a device address: the address is obtained per device with cudaGetSymbolAddress and handed to the kernels.
+static __device__ __align__(256) unsigned char g_static_scratch[EAS_STATIC_WORKSPACE_BYTES];
+
+namespace {
+constexpr int kMaxDevices = 64;
+std::mutex g_static_mutex;
+unsigned char* g_static_ptr[kMaxDevices] = {};   // device address of g_static_scratch on each device, once known
+}  // namespace
+
+extern "C" eas_status eas_encode_microbatch_static(eas_encoder* e, const eas_packed_inputs* in, const int32_t* cu_dev,
+                                                   int32_t sm_budget, void* stream_v, void* out_embeddings) {
+  int dev = 0;
+  CUDA_TRY(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= kMaxDevices) return fail(EAS_ERR_UNSUPPORTED, "device ordinal %d", dev);
+  unsigned char* base = nullptr;
+  {
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    if (g_static_ptr[dev] == nullptr) {
+      // first call on this device (the device is current): look the symbol's device address up once
+      void* sym = nullptr;
+      CUDA_TRY(cudaGetSymbolAddress(&sym, g_static_scratch));
+      if (sym == nullptr) return fail(EAS_ERR_CUDA, "cudaGetSymbolAddress returned a null address");
+      g_static_ptr[dev] = static_cast<unsigned char*>(sym);
+    }
+    base = g_static_ptr[dev];
+  }
+  // the forward pass wants its scratch on a 1024-byte boundary; the array itself is only 256-byte aligned
+  const uintptr_t aligned = (reinterpret_cast<uintptr_t>(base) + 1023) & ~uintptr_t(1023);
+  const size_t usable = EAS_STATIC_WORKSPACE_BYTES - (aligned - reinterpret_cast<uintptr_t>(base));
+  if (e != nullptr && in != nullptr && in->cu_seqlens_host != nullptr && in->n_items >= 1 && in->n_items <= EAS_MAX_ITEMS) {
+    const int64_t T = in->cu_seqlens_host[in->n_items];
+    if (T > 0) {
+      const size_t need = make_plan(e, T, in->n_items).total;
+      if (need > usable)
+        return fail(EAS_ERR_WORKSPACE,
+                    "micro-batch needs %zu bytes of scratch but the built-in scratch holds %zu: use eas_encode_microbatch "
+                    "with a caller-allocated workspace, or send fewer / smaller items", need, usable);
+    }
+  }
+  return encode_impl(e, in, reinterpret_cast<void*>(aligned), usable, cu_dev, sm_budget, stream_v, out_embeddings);
 }
 
 extern "C" eas_status eas_encoder_enable_timing(eas_encoder* e, int32_t on) {
