@@ -70,11 +70,11 @@ static eas_status make_tmap(CUtensorMap* m, const void* base, int rank, const ui
   return EAS_OK;
 }
 
-// W [N, K] row-major -> 2-D map, box 64 x 256
-static eas_status make_w_tmap(CUtensorMap* m, const void* w, int64_t N, int64_t K) {
+// W [N, K] row-major -> 2-D map, box 64 x `box_rows` (256: one CTA loads the whole weight tile; 128: half of it)
+static eas_status make_w_tmap(CUtensorMap* m, const void* w, int64_t N, int64_t K, uint32_t box_rows) {
   const uint64_t dims[2] = {static_cast<uint64_t>(K), static_cast<uint64_t>(N)};
   const uint64_t strides[1] = {static_cast<uint64_t>(K) * 2};
-  const uint32_t box[2] = {kBK, kBN};
+  const uint32_t box[2] = {kBK, box_rows};
   return make_tmap(m, w, 2, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B);
 }
 // A as {run, phase, rows}: a plain [M, K] matrix is {K, 1, M}; a k=3 convolution over rows of width C with row
@@ -107,7 +107,8 @@ struct Linear {
   const bf16* w = nullptr;   // [N, K] (possibly re-laid)
   const bf16* b = nullptr;   // [N]
   int N = 0, K = 0;
-  CUtensorMap tmap;
+  CUtensorMap tmap;        // box of 256 weight rows
+  CUtensorMap tmap_half;   // box of 128 weight rows (CTA-pair kernel)
 };
 struct Layer {
   const bf16 *n1g = nullptr, *n1b = nullptr, *n2g = nullptr, *n2b = nullptr;
@@ -240,14 +241,36 @@ static eas_status relayout(bf16* dst, const bf16* src, const bf16* src2, long lo
     if (s_ != EAS_OK) return s_; \
   } while (0)
 
-static eas_status finish_linear(Linear& L) { return make_w_tmap(&L.tmap, L.w, L.N, L.K); }
+static eas_status finish_linear(Linear& L) {
+  EAS_TRY(make_w_tmap(&L.tmap, L.w, L.N, L.K, kBN));
+  return make_w_tmap(&L.tmap_half, L.w, L.N, L.K, kBN / 2);
+}
 
+typedef void (*GemmKernel)(GemmParams);
+static GemmKernel gemm_kernel_for(int act, int out_fp32, int ctas) {
+  if (ctas == 2) {
+    if (act == ACT_NONE && !out_fp32) return gemm_kernel<ACT_NONE, OUT_BF16, 2>;
+    if (act == ACT_GELU && !out_fp32) return gemm_kernel<ACT_GELU, OUT_BF16, 2>;
+    if (act == ACT_SWIGLU && !out_fp32) return gemm_kernel<ACT_SWIGLU, OUT_BF16, 2>;
+    if (act == ACT_NONE && out_fp32) return gemm_kernel<ACT_NONE, OUT_F32, 2>;
+    if (act == ACT_GELU && out_fp32) return gemm_kernel<ACT_GELU, OUT_F32, 2>;
+  } else {
+    if (act == ACT_NONE && !out_fp32) return gemm_kernel<ACT_NONE, OUT_BF16, 1>;
+    if (act == ACT_GELU && !out_fp32) return gemm_kernel<ACT_GELU, OUT_BF16, 1>;
+    if (act == ACT_SWIGLU && !out_fp32) return gemm_kernel<ACT_SWIGLU, OUT_BF16, 1>;
+    if (act == ACT_NONE && out_fp32) return gemm_kernel<ACT_NONE, OUT_F32, 1>;
+    if (act == ACT_GELU && out_fp32) return gemm_kernel<ACT_GELU, OUT_F32, 1>;
+  }
+  return nullptr;
+}
 static eas_status set_kernel_attributes() {
-  CUDA_TRY(cudaFuncSetAttribute(gemm_kernel<ACT_NONE, OUT_BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmemBytes));
-  CUDA_TRY(cudaFuncSetAttribute(gemm_kernel<ACT_GELU, OUT_BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmemBytes));
-  CUDA_TRY(cudaFuncSetAttribute(gemm_kernel<ACT_SWIGLU, OUT_BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmemBytes));
-  CUDA_TRY(cudaFuncSetAttribute(gemm_kernel<ACT_NONE, OUT_F32>, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmemBytes));
-  CUDA_TRY(cudaFuncSetAttribute(gemm_kernel<ACT_GELU, OUT_F32>, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmemBytes));
+  for (int ctas = 1; ctas <= 2; ++ctas)
+    for (int act = 0; act < 3; ++act)
+      for (int f32 = 0; f32 < 2; ++f32) {
+        GemmKernel k = gemm_kernel_for(act, f32, ctas);
+        if (k != nullptr)
+          CUDA_TRY(cudaFuncSetAttribute(reinterpret_cast<const void*>(k), cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmemBytes));
+      }
   return EAS_OK;
 }
 
@@ -486,14 +509,16 @@ static eas_status launch_gemm(const GemmCall& g, int budget, cudaStream_t stream
   const Linear& L = *g.lin;
   if (g.M <= 0) return EAS_OK;
   if (L.N % 32 != 0 || g.a_run % kBK != 0) return fail(EAS_ERR_UNSUPPORTED, "GEMM needs N %% 32 == 0 and K %% 64 == 0 (N=%d, K=%lld)", L.N, static_cast<long long>(g.a_run));
+  // CTA pairs (two SMs on one 256x256 tile, each loading half of the weight tile) whenever two SMs are available
+  const int ctas = budget >= 2 ? 2 : 1;
   GemmParams p{};
   EAS_TRY(make_a_tmap(&p.tma_a, g.A, g.a_run, g.a_row_elems, g.conv_stride, g.a_rows));
-  p.tma_b = L.tmap;
+  p.tma_b = ctas == 2 ? L.tmap_half : L.tmap;
   p.M = g.M; p.N = L.N;
   p.kb_per_tap = static_cast<int>(g.a_run / kBK);
   p.k_blocks = p.kb_per_tap * g.taps;
   p.conv_stride = g.conv_stride;
-  p.m_blocks = (g.M + kBM - 1) / kBM;
+  p.m_blocks = (g.M + kBM * ctas - 1) / (kBM * ctas);
   p.n_blocks = (L.N + kBN - 1) / kBN;
   p.bias = L.b;
   p.out = g.out; p.ldo = g.ldo; p.resid = g.resid;
@@ -507,16 +532,21 @@ static eas_status launch_gemm(const GemmCall& g, int budget, cudaStream_t stream
     EAS_TRY(make_out_tmap(&p.tma_out, g.out, g.out_fp32 != 0, out_cols, g.ldo, g.M));
   }
   const int tiles = p.m_blocks * p.n_blocks;
-  const int grid = std::min(budget, tiles);
-  void (*kern)(GemmParams) = nullptr;
-  if (g.act == ACT_NONE && !g.out_fp32) kern = gemm_kernel<ACT_NONE, OUT_BF16>;
-  else if (g.act == ACT_GELU && !g.out_fp32) kern = gemm_kernel<ACT_GELU, OUT_BF16>;
-  else if (g.act == ACT_SWIGLU && !g.out_fp32) kern = gemm_kernel<ACT_SWIGLU, OUT_BF16>;
-  else if (g.act == ACT_NONE && g.out_fp32) kern = gemm_kernel<ACT_NONE, OUT_F32>;
-  else if (g.act == ACT_GELU && g.out_fp32) kern = gemm_kernel<ACT_GELU, OUT_F32>;
-  else return fail(EAS_ERR_UNSUPPORTED, "no GEMM epilogue for act=%d out_fp32=%d", g.act, g.out_fp32);
-  kern<<<grid, kGemmThreads, kGemmSmemBytes, stream>>>(p);
-  CUDA_TRY(cudaGetLastError());
+  GemmKernel kern = gemm_kernel_for(g.act, g.out_fp32, ctas);
+  if (kern == nullptr) return fail(EAS_ERR_UNSUPPORTED, "no GEMM epilogue for act=%d out_fp32=%d", g.act, g.out_fp32);
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3(static_cast<unsigned>(std::min(budget / ctas, tiles) * ctas), 1, 1);
+  cfg.blockDim = dim3(kGemmThreads, 1, 1);
+  cfg.dynamicSmemBytes = kGemmSmemBytes;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = static_cast<unsigned>(ctas);
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, p));
   return EAS_OK;
 }
 

@@ -15,16 +15,21 @@
 namespace eas {
 
 constexpr int kBM = 128, kBN = 256, kBK = 64;
-constexpr int kStages = 4;
 constexpr int kEpiWarps = 8;
 constexpr int kGemmThreads = 64 + 32 * kEpiWarps;
-constexpr int kABytes = kBM * kBK * 2;            // 16 KB
-constexpr int kBBytes = kBN * kBK * 2;            // 32 KB
-constexpr int kStageBytes = kABytes + kBBytes;    // 48 KB
-constexpr int kStagingOff = kStages * kStageBytes;             // 8 epilogue warps x 4 KB output staging (TMA store source)
+constexpr int kABytes = kBM * kBK * 2;            // 16 KB: 128 rows of A
+// one CTA per tile: a stage holds A (16 KB) + the whole 256-row weight tile (32 KB), 4 stages;
+// CTA pair per 256x256 tile: a stage holds A (16 KB) + this CTA's 128 weight rows (16 KB), 6 stages
+template <int CTAS> struct GemmCfg {
+  static constexpr int kBBytes = (kBN / CTAS) * kBK * 2;
+  static constexpr int kStageBytes = kABytes + kBBytes;
+  static constexpr int kStages = CTAS == 2 ? 6 : 4;
+};
+constexpr int kMaxStages = 6;
+constexpr int kStagingOff = 4 * 49152;                         // == 6 * 32768; 8 epilogue warps x 4 KB output staging (TMA store source)
 constexpr int kBiasOff = kStagingOff + kEpiWarps * 4096;       // 2 x 256 fp32 bias values of the current tiles
 constexpr int kBarOff = kBiasOff + 2 * 256 * 4;
-constexpr int kGemmSmemBytes = kBarOff + 128 /*barriers*/ + 896 /*alignment slack: the base is 128-byte aligned at least*/;
+constexpr int kGemmSmemBytes = kBarOff + 192 /*barriers*/ + 832 /*alignment slack*/;
 static_assert(kGemmSmemBytes <= 232448, "exceeds the 227 KB shared memory of an SM");
 constexpr int kTmemCols = 512;
 constexpr int kPanelM = 8;                        // m-blocks per rasterisation panel (L2 reuse of W tiles)
@@ -34,14 +39,14 @@ enum { OUT_BF16 = 0, OUT_F32 = 1 };
 
 struct alignas(64) GemmParams {
   CUtensorMap tma_a;      // 3-D: {K-run, phase, rows}; box {64, 1, 128}
-  CUtensorMap tma_b;      // 2-D: {K, N}; box {64, 256}
+  CUtensorMap tma_b;      // 2-D: {K, N}; box {64, 256} (one CTA per tile) or {64, 128} (CTA pair)
   CUtensorMap tma_out;    // 2-D over out: box {64 bf16 | 32 fp32, 32 rows}, 128-byte swizzle (valid if use_tma_out)
   int use_tma_out;        // 1: epilogue stages 32-row sub-tiles in shared memory and stores them with TMA
   int M, N;               // rows of A walked by tiles; rows of W
   int k_blocks;           // K / 64 (K padded with zeros by the caller or by TMA fill)
   int kb_per_tap;         // k-blocks per convolution tap (== k_blocks for a plain GEMM)
   int conv_stride;        // 1 for a plain GEMM; row stride of a convolution otherwise
-  int m_blocks, n_blocks;
+  int m_blocks, n_blocks; // m_blocks counts 128-row blocks (one CTA per tile) or 256-row blocks (CTA pair)
   const bf16* bias;       // [N] (for SWIGLU: interleaved gate/up like the W rows)
   void* out;              // bf16 or fp32 [*, ldo]
   long long ldo;          // leading dimension of out (elements)
@@ -65,27 +70,32 @@ __device__ __forceinline__ void tile_coords(int tile, int m_blocks, int n_blocks
   mb = panel * kPanelM + (within - nb * rows_here);
 }
 
-template <int ACT, int OUT>
+template <int ACT, int OUT, int CTAS>
 __global__ void __launch_bounds__(kGemmThreads, 1) gemm_kernel(const __grid_constant__ GemmParams p) {
+  constexpr int kStages = GemmCfg<CTAS>::kStages;
+  constexpr int kStageBytes = GemmCfg<CTAS>::kStageBytes;
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   // 1024-byte alignment: the 128-byte swizzle pattern repeats every 8 rows of 128 bytes
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kBarOff);
-  uint64_t* full_bar = bars;                    // [kStages]  TMA -> MMA
-  uint64_t* empty_bar = bars + kStages;         // [kStages]  MMA -> TMA
-  uint64_t* acc_full = bars + 2 * kStages;      // [2]        MMA -> epilogue
-  uint64_t* acc_empty = bars + 2 * kStages + 2; // [2]        epilogue -> MMA
-  uint64_t* bias_bar = bars + 2 * kStages + 4;  // [2]        epilogue warps: bias values staged
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kStages + 6);
+  uint64_t* full_bar = bars;                       // [kStages]  TMA -> MMA (pair: the leader's copy collects both CTAs' bytes)
+  uint64_t* empty_bar = bars + kMaxStages;         // [kStages]  MMA -> TMA (pair: signalled in both CTAs)
+  uint64_t* acc_full = bars + 2 * kMaxStages;      // [2]        MMA -> epilogue (pair: signalled in both CTAs)
+  uint64_t* acc_empty = bars + 2 * kMaxStages + 2; // [2]        epilogue -> MMA (pair: both CTAs' warps arrive at the leader)
+  uint64_t* bias_bar = bars + 2 * kMaxStages + 4;  // [2]        epilogue warps: bias values staged
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kMaxStages + 6);
   volatile uint32_t* abort_flag = tmem_slot + 1;
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
   const int num_tiles = p.m_blocks * p.n_blocks;
+  const int cta_rank = CTAS == 2 ? static_cast<int>(cluster_ctarank()) : 0;
+  const int first_tile = blockIdx.x / CTAS;        // both CTAs of a pair walk the same tiles
+  const int tile_step = gridDim.x / CTAS;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
-    for (int a = 0; a < 2; ++a) { mbar_init(&acc_full[a], 1); mbar_init(&acc_empty[a], kEpiWarps); mbar_init(&bias_bar[a], kEpiWarps); }
+    for (int a = 0; a < 2; ++a) { mbar_init(&acc_full[a], 1); mbar_init(&acc_empty[a], kEpiWarps * CTAS); mbar_init(&bias_bar[a], kEpiWarps); }
     *abort_flag = 0;
     mbar_fence_init();
     tma_prefetch_desc(&p.tma_a);
@@ -93,11 +103,12 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_kernel(const __grid_cons
     if (p.use_tma_out) tma_prefetch_desc(&p.tma_out);
   }
   if (warp == 1) {
-    tmem_alloc(tmem_slot, kTmemCols);
-    tmem_relinquish();
+    if (CTAS == 2) { tmem_alloc_pair(tmem_slot, kTmemCols); tmem_relinquish_pair(); }
+    else { tmem_alloc(tmem_slot, kTmemCols); tmem_relinquish(); }
   }
   tc_fence_before_sync();
   __syncthreads();
+  if (CTAS == 2) cluster_sync_all();               // the peer's barriers are initialised before anything signals them
   tc_fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
 
@@ -106,20 +117,28 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_kernel(const __grid_cons
     if (lane == 0) {
       uint32_t it = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
-        int mb, nb;
-        tile_coords(tile, p.m_blocks, p.n_blocks, mb, nb);
+      for (int tile = first_tile; tile < num_tiles && ok; tile += tile_step) {
+        int mg, nb;
+        tile_coords(tile, p.m_blocks, p.n_blocks, mg, nb);
+        const int mb = mg * CTAS + cta_rank;       // this CTA's 128-row block
         for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
           const int s = it % kStages;
           const uint32_t ph = (it / kStages) & 1u;
           if (!mbar_wait(&empty_bar[s], ph ^ 1u, abort_flag)) { ok = false; break; }
           uint8_t* sa = smem + s * kStageBytes;
           uint8_t* sb = sa + kABytes;
-          mbar_expect_tx(&full_bar[s], kStageBytes);
           const int tap = kb / p.kb_per_tap;
           const int kx = (kb - tap * p.kb_per_tap) * kBK;
-          tma_load_3d(sa, &p.tma_a, &full_bar[s], kx, tap % p.conv_stride, mb * kBM + tap / p.conv_stride);
-          tma_load_2d(sb, &p.tma_b, &full_bar[s], kb * kBK, nb * kBN);
+          if (CTAS == 2) {
+            // both CTAs' loads complete on the leader's barrier; the leader announces the bytes of both
+            if (cta_rank == 0) mbar_expect_tx(&full_bar[s], 2 * kStageBytes);
+            tma_load_3d_pair(sa, &p.tma_a, &full_bar[s], kx, tap % p.conv_stride, mb * kBM + tap / p.conv_stride);
+            tma_load_2d_pair(sb, &p.tma_b, &full_bar[s], kb * kBK, nb * kBN + cta_rank * (kBN / 2));
+          } else {
+            mbar_expect_tx(&full_bar[s], kStageBytes);
+            tma_load_3d(sa, &p.tma_a, &full_bar[s], kx, tap % p.conv_stride, mb * kBM + tap / p.conv_stride);
+            tma_load_2d(sb, &p.tma_b, &full_bar[s], kb * kBK, nb * kBN);
+          }
         }
       }
       if (!ok) {
@@ -132,11 +151,11 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_kernel(const __grid_cons
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ UMMA issuer
-    if (lane == 0) {
-      constexpr uint32_t idesc = make_idesc_bf16(kBM, kBN, 0, 0);
+    if (lane == 0 && cta_rank == 0) {
+      constexpr uint32_t idesc = make_idesc_bf16(kBM * CTAS, kBN, 0, 0);
       uint32_t it = 0, tcount = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++tcount) {
+      for (int tile = first_tile; tile < num_tiles && ok; tile += tile_step, ++tcount) {
         const uint32_t acc = tcount & 1u;
         const uint32_t acc_ph = (tcount >> 1) & 1u;
         if (!mbar_wait(&acc_empty[acc], acc_ph ^ 1u, abort_flag)) { ok = false; break; }
@@ -154,11 +173,15 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_kernel(const __grid_cons
 #pragma unroll
           for (int k = 0; k < kBK / 16; ++k) {
             // advancing 16 bf16 = 32 bytes along K inside the swizzle atom: +2 in the (>>4) address field
-            umma_bf16_ss(tmem_d, adesc + 2 * k, bdesc + 2 * k, idesc, (kb | k) != 0);
+            if (CTAS == 2) umma_bf16_ss_pair(tmem_d, adesc + 2 * k, bdesc + 2 * k, idesc, (kb | k) != 0);
+            else umma_bf16_ss(tmem_d, adesc + 2 * k, bdesc + 2 * k, idesc, (kb | k) != 0);
           }
-          umma_commit(&empty_bar[s]);           // frees the stage once these UMMAs have read it
+          // frees the stage (in both CTAs of a pair) once these UMMAs have read it
+          if (CTAS == 2) umma_commit_pair_multicast(&empty_bar[s], 3); else umma_commit(&empty_bar[s]);
         }
-        if (ok) umma_commit(&acc_full[acc]);    // accumulator complete
+        if (ok) {                               // accumulator complete
+          if (CTAS == 2) umma_commit_pair_multicast(&acc_full[acc], 3); else umma_commit(&acc_full[acc]);
+        }
       }
     }
   } else {
@@ -168,9 +191,17 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_kernel(const __grid_cons
     const int half = ew >> 2;                   // which 128 accumulator columns
     uint32_t tcount = 0;
     bool ok = true;
-    for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++tcount) {
-      int mb, nb;
-      tile_coords(tile, p.m_blocks, p.n_blocks, mb, nb);
+    auto release_accumulator = [&](uint32_t acc) {   // this warp has read its part of the accumulator
+      tc_fence_before_sync();
+      __syncwarp();
+      if (lane == 0) {
+        if (CTAS == 2) mbar_arrive_cluster(&acc_empty[acc], 0); else mbar_arrive(&acc_empty[acc]);
+      }
+    };
+    for (int tile = first_tile; tile < num_tiles && ok; tile += tile_step, ++tcount) {
+      int mg, nb;
+      tile_coords(tile, p.m_blocks, p.n_blocks, mg, nb);
+      const int mb = mg * CTAS + cta_rank;
       const uint32_t acc = tcount & 1u;
       const uint32_t acc_ph = (tcount >> 1) & 1u;
       if (p.use_tma_out) {
@@ -291,9 +322,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_kernel(const __grid_cons
             if (col0 < p.N) store_subtile(col0);
           }
         }
-        tc_fence_before_sync();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&acc_empty[acc]);
+        release_accumulator(acc);
         continue;
       }
 
@@ -405,9 +434,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_kernel(const __grid_cons
         }
       }
       // all TMEM reads of this warp are complete (wait::ld above): hand the accumulator back
-      tc_fence_before_sync();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&acc_empty[acc]);
+      release_accumulator(acc);
     }
     // bulk stores still reading the staging buffer must finish before the CTA's shared memory is released
     if (p.use_tma_out && lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
@@ -415,9 +442,10 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_kernel(const __grid_cons
 
   tc_fence_before_sync();
   __syncthreads();
+  if (CTAS == 2) cluster_sync_all();               // no CTA of the pair retires while the other may still signal it
   if (warp == 1) {
     tc_fence_after_sync();
-    tmem_dealloc(tmem_base, kTmemCols);
+    if (CTAS == 2) tmem_dealloc_pair(tmem_base, kTmemCols); else tmem_dealloc(tmem_base, kTmemCols);
   }
   if (threadIdx.x == 0 && *abort_flag) atomicCAS(p.status, DEV_OK, DEV_ERR_WAIT_TIMEOUT);
 }
