@@ -61,6 +61,8 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attn_mma_kernel(const __grid_
   bf16* sV = sK + 2 * kAttnBKV * LDS;      // [2][64][LDS]
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  pdl_launch_dependents();
+  pdl_wait();
 
   for (int unit = blockIdx.x; unit < p.total_units; unit += gridDim.x) {
     // decode (item, head, q-tile); q-tile varies fastest so that neighbours share K and V in L2

@@ -181,6 +181,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_tc_kernel(const __grid_con
   __syncthreads();
   tc_fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
+  pdl_launch_dependents();
+  pdl_wait();
   // TMEM columns: S_A [0,128)  S_B [128,256)  O_A [256,256+HD)  O_B [384,384+HD)
 
   auto q_tile = [&](int buf, int t) { return smem + L::kQOff + (buf * 2 + t) * L::kTileBytes; };

@@ -482,6 +482,34 @@ extern "C" int64_t eas_encoder_out_rows(const eas_encoder* enc, const int32_t* c
 }
 
 // ------------------------------------------------------------------------------------ launch helpers
+// Every per-call kernel is launched with programmatic stream serialization: it may be set up while its
+// predecessor in the stream drains and waits (griddepcontrol.wait) before touching any data.
+template <typename Params>
+static eas_status launch_kernel(void (*kern)(Params), int grid, int block, size_t smem, cudaStream_t stream, const Params& params,
+                                int cluster = 1) {
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3(static_cast<unsigned>(grid), 1, 1);
+  cfg.blockDim = dim3(static_cast<unsigned>(block), 1, 1);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[2];
+  int n = 0;
+  attr[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[n].val.programmaticStreamSerializationAllowed = 1;
+  ++n;
+  if (cluster > 1) {
+    attr[n].id = cudaLaunchAttributeClusterDimension;
+    attr[n].val.clusterDim.x = static_cast<unsigned>(cluster);
+    attr[n].val.clusterDim.y = 1;
+    attr[n].val.clusterDim.z = 1;
+    ++n;
+  }
+  cfg.attrs = attr;
+  cfg.numAttrs = n;
+  CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, params));
+  return EAS_OK;
+}
+
 namespace {
 struct GemmCall {
   const void* A = nullptr;   // bf16
@@ -534,20 +562,7 @@ static eas_status launch_gemm(const GemmCall& g, int budget, cudaStream_t stream
   const int tiles = p.m_blocks * p.n_blocks;
   GemmKernel kern = gemm_kernel_for(g.act, g.out_fp32, ctas);
   if (kern == nullptr) return fail(EAS_ERR_UNSUPPORTED, "no GEMM epilogue for act=%d out_fp32=%d", g.act, g.out_fp32);
-  cudaLaunchConfig_t cfg{};
-  cfg.gridDim = dim3(static_cast<unsigned>(std::min(budget / ctas, tiles) * ctas), 1, 1);
-  cfg.blockDim = dim3(kGemmThreads, 1, 1);
-  cfg.dynamicSmemBytes = kGemmSmemBytes;
-  cfg.stream = stream;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeClusterDimension;
-  attr[0].val.clusterDim.x = static_cast<unsigned>(ctas);
-  attr[0].val.clusterDim.y = 1;
-  attr[0].val.clusterDim.z = 1;
-  cfg.attrs = attr;
-  cfg.numAttrs = 1;
-  CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, p));
-  return EAS_OK;
+  return launch_kernel(kern, std::min(budget / ctas, tiles) * ctas, kGemmThreads, kGemmSmemBytes, stream, p, ctas);
 }
 
 template <int KIND, bool F32>
@@ -560,7 +575,7 @@ static eas_status launch_norm_nv(const NormParams& p, int budget, cudaStream_t s
       CUDA_TRY(cudaFuncSetAttribute(norm_kernel<NV_, KIND, F32>, cudaFuncAttributeMaxDynamicSharedMemorySize, kOnePerSmSmem)); \
       attr_set = true;                                                                                             \
     }                                                                                                              \
-    norm_kernel<NV_, KIND, F32><<<std::min(budget, (p.rows + 15) / 16), 512, kOnePerSmSmem, stream>>>(p);          \
+    EAS_TRY(launch_kernel(norm_kernel<NV_, KIND, F32>, std::min(budget, (p.rows + 15) / 16), 512, kOnePerSmSmem, stream, p)); \
     break;                                                                                                         \
   }
   switch (nv) {
@@ -618,11 +633,9 @@ static eas_status launch_attention_mma(const bf16* qkv, bf16* out, const int32_t
     attr_set = true;
   }
   static_assert(attn_mma_smem_bytes<80>() <= kOnePerSmSmem, "attention tile does not fit");
-  if (hd == 64) attn_mma_kernel<64><<<grid, kAttnThreads, kOnePerSmSmem, stream>>>(ap);
-  else if (hd == 80) attn_mma_kernel<80><<<grid, kAttnThreads, kOnePerSmSmem, stream>>>(ap);
-  else return fail(EAS_ERR_UNSUPPORTED, "head_dim %d", hd);
-  CUDA_TRY(cudaGetLastError());
-  return EAS_OK;
+  if (hd == 64) return launch_kernel(attn_mma_kernel<64>, grid, kAttnThreads, kOnePerSmSmem, stream, ap);
+  if (hd == 80) return launch_kernel(attn_mma_kernel<80>, grid, kAttnThreads, kOnePerSmSmem, stream, ap);
+  return fail(EAS_ERR_UNSUPPORTED, "head_dim %d", hd);
 }
 
 static eas_status launch_attention_tc(const bf16* qkv, bf16* out, const int32_t* cu, int n_items, int H, int hd, int budget,
@@ -651,11 +664,9 @@ static eas_status launch_attention_tc(const bf16* qkv, bf16* out, const int32_t*
     CUDA_TRY(cudaFuncSetAttribute(attn_tc_kernel<80>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttnTcSmem<80>::kBytes));
     attr_set = true;
   }
-  if (hd == 64) attn_tc_kernel<64><<<grid, kTcThreads, AttnTcSmem<64>::kBytes, stream>>>(ap);
-  else if (hd == 80) attn_tc_kernel<80><<<grid, kTcThreads, AttnTcSmem<80>::kBytes, stream>>>(ap);
-  else return fail(EAS_ERR_UNSUPPORTED, "head_dim %d", hd);
-  CUDA_TRY(cudaGetLastError());
-  return EAS_OK;
+  if (hd == 64) return launch_kernel(attn_tc_kernel<64>, grid, kTcThreads, AttnTcSmem<64>::kBytes, stream, ap);
+  if (hd == 80) return launch_kernel(attn_tc_kernel<80>, grid, kTcThreads, AttnTcSmem<80>::kBytes, stream, ap);
+  return fail(EAS_ERR_UNSUPPORTED, "head_dim %d", hd);
 }
 
 static eas_status launch_attention(const bf16* qkv, bf16* out, const int32_t* cu, int n_items, int H, int hd, int budget,
@@ -759,8 +770,7 @@ static eas_status encode_impl(eas_encoder* e, const eas_packed_inputs* in, void*
     pp.rope_cs = rope; pp.x = x; pp.cls = e->cls; pp.pos = e->pos;
     pp.conv1_row_map = conv1_map; pp.n_conv1_rows = static_cast<int>(pl.padded_rows);
     pp.status = status;
-    prep_kernel<<<budget, 256, 0, stream>>>(pp);
-    CUDA_TRY(cudaGetLastError());
+    EAS_TRY(launch_kernel(prep_kernel, budget, 256, 0, stream, pp));
     ++launches;
   }
 
@@ -773,8 +783,7 @@ static eas_status encode_impl(eas_encoder* e, const eas_packed_inputs* in, void*
     static bool attr_set = false;
     if (!attr_set) { CUDA_TRY(cudaFuncSetAttribute(audio_stage_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kOnePerSmSmem)); attr_set = true; }
     EAS_TRY(mark(e, EAS_KC_EMBED_GATHER, stream));
-    audio_stage_kernel<<<budget, 512, kOnePerSmSmem, stream>>>(sp);
-    CUDA_TRY(cudaGetLastError());
+    EAS_TRY(launch_kernel(audio_stage_kernel, budget, 512, kOnePerSmSmem, stream, sp));
     ++launches;
     GemmCall g1;   // conv1 (k=3, stride 1) + GELU -> padded h1
     g1.A = mel_pad; g1.a_run = c.in_channels; g1.a_row_elems = c.in_channels; g1.conv_stride = 1; g1.taps = 3;
@@ -798,8 +807,7 @@ static eas_status encode_impl(eas_encoder* e, const eas_packed_inputs* in, void*
     static bool attr_set = false;
     if (!attr_set) { CUDA_TRY(cudaFuncSetAttribute(im2col_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kOnePerSmSmem)); attr_set = true; }
     EAS_TRY(mark(e, EAS_KC_EMBED_GATHER, stream));
-    im2col_kernel<<<budget, 512, kOnePerSmSmem, stream>>>(ip);
-    CUDA_TRY(cudaGetLastError());
+    EAS_TRY(launch_kernel(im2col_kernel, budget, 512, kOnePerSmSmem, stream, ip));
     ++launches;
     GemmCall g;
     g.A = embed_a; g.a_run = e->embed_k_pad; g.a_row_elems = e->embed_k_pad; g.a_rows = pl.embed_rows; g.M = static_cast<int>(pl.embed_rows);

@@ -61,6 +61,8 @@ __global__ void __launch_bounds__(512, 1) norm_kernel(const NormParams p) {
     }
   }
   const float inv_d = 1.0f / static_cast<float>(p.d);
+  pdl_launch_dependents();
+  pdl_wait();
   for (int row = blockIdx.x * warps_per_cta + warp; row < p.rows; row += gridDim.x * warps_per_cta) {
     const long long src = p.src_rows ? p.src_rows[row] : row;
     const float4* xr = reinterpret_cast<const float4*>(p.x + src * p.d);
@@ -120,6 +122,8 @@ struct Im2colParams {
 __global__ void __launch_bounds__(512, 1) im2col_kernel(const __grid_constant__ Im2colParams p) {
   const int P = p.patch;
   const long long total = static_cast<long long>(p.n_patches) * p.k_pad;
+  pdl_launch_dependents();
+  pdl_wait();
   for (long long idx = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x; idx < total;
        idx += static_cast<long long>(gridDim.x) * blockDim.x) {
     const int m = static_cast<int>(idx / p.k_pad);
@@ -186,6 +190,8 @@ __global__ void __launch_bounds__(256) prep_kernel(const __grid_constant__ PrepP
   const int gtid = blockIdx.x * blockDim.x + threadIdx.x;
   const int gsz = gridDim.x * blockDim.x;
   const int n = p.items.n_items;
+  pdl_launch_dependents();
+  pdl_wait();
   if (p.cu_seqlens_dev != nullptr) {
     for (int i = gtid; i <= n; i += gsz)
       if (p.cu_seqlens_dev[i] != p.items.tok_start[i]) atomicCAS(p.status, DEV_OK, DEV_ERR_CU_SEQLENS_MISMATCH);
@@ -272,6 +278,8 @@ struct AudioStageParams {
 __global__ void __launch_bounds__(512, 1) audio_stage_kernel(const __grid_constant__ AudioStageParams p) {
   const long long total = static_cast<long long>(p.padded_rows) * p.n_mel;
   const long long gsz = static_cast<long long>(gridDim.x) * blockDim.x;
+  pdl_launch_dependents();
+  pdl_wait();
   for (long long idx = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x; idx < total; idx += gsz) {
     const int m = static_cast<int>(idx / p.n_mel);
     const int c = static_cast<int>(idx - static_cast<long long>(m) * p.n_mel);

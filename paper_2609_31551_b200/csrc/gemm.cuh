@@ -111,6 +111,8 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_kernel(const __grid_cons
   if (CTAS == 2) cluster_sync_all();               // the peer's barriers are initialised before anything signals them
   tc_fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
+  pdl_launch_dependents();   // the next kernel may set itself up while this one runs
+  pdl_wait();                // everything before this kernel in the stream is complete and visible
 
   if (warp == 0) {
     // ------------------------------------------------------------------ producer
