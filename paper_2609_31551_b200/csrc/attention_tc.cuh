@@ -119,6 +119,16 @@ __device__ __forceinline__ void setmaxnreg_inc() { asm volatile("setmaxnreg.inc.
 template <int N>
 __device__ __forceinline__ void setmaxnreg_dec() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N)); }
 
+#ifdef EAS_ATTN_PROFILE
+// phase timestamps of the first softmax warp of each warpgroup in CTA 0 (profiling builds only)
+__device__ unsigned long long g_attn_dbg[2 * 64 * 12];
+#define ATTN_STAMP(k) do { if (blockIdx.x == 0 && quarter == 0 && lane == 0 && n < 64) g_attn_dbg[(w * 64 + n) * 12 + (k)] = clock64(); } while (0)
+#define ATTN_STAMP_PREV(k) do { if (blockIdx.x == 0 && quarter == 0 && lane == 0 && n >= 1 && n <= 64) g_attn_dbg[(w * 64 + n - 1) * 12 + (k)] = clock64(); } while (0)
+#else
+#define ATTN_STAMP(k) do { } while (0)
+#define ATTN_STAMP_PREV(k) do { } while (0)
+#endif
+
 struct UnitInfo {
   int head, q0, S, n_kv, n_q;
   long long row0;
@@ -270,31 +280,54 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_tc_kernel(const __grid_con
         ++n_pv[w];
       };
 
+      bool pre_issued[2] = {false, false};       // S(w, 0) of this unit was already issued at the end of the previous one
       for (int unit = blockIdx.x; unit < p.total_units && ok; unit += gridDim.x, ++u_cnt) {
         const UnitInfo u = decode_unit(p, unit);
         const int qb = u_cnt & 1;
+        const bool has_next = unit + static_cast<int>(gridDim.x) < p.total_units;
+        UnitInfo un = u;
+        if (has_next) un = decode_unit(p, unit + gridDim.x);
         if (!mbar_wait(&q_full[qb], (u_cnt >> 1) & 1u, abort_flag)) { ok = false; break; }
         {
           const int s = kv_it % NST;
           if (!mbar_wait(&k_full[s], (kv_it / NST) & 1u, abort_flag)) { ok = false; break; }
           tc_fence_after_sync();
-          for (int w = 0; w < u.n_q; ++w) issue_s(w, qb, s);
+#pragma unroll
+          for (int w = 0; w < 2; ++w) if (w < u.n_q && !pre_issued[w]) issue_s(w, qb, s);
+          pre_issued[0] = pre_issued[1] = false;
         }
+        bool next_q_ready = false;
         for (int j = 0; j < u.n_kv && ok; ++j, ++kv_it) {
           const int s = kv_it % NST;
           const int sn = (kv_it + 1) % NST;
-          for (int w = 0; w < u.n_q; ++w) {
+          const bool last = j + 1 == u.n_kv;
+#pragma unroll
+          for (int w = 0; w < 2; ++w) {
+            if (w >= u.n_q) break;
             // P(w, j) is in shared memory, S(w) has been read, O(w) has been rescaled if it had to be
             if (!mbar_wait(&p_ready[w], (n_pv[w]) & 1u, abort_flag)) { ok = false; break; }
             tc_fence_after_sync();
-            if (j + 1 < u.n_kv) {
+            // next scores first (the softmax of the next tile overlaps P V of this one); after the unit's last
+            // tile the next scores are the first tile of the NEXT unit, so the pipeline never drains
+            if (!last) {
               if (w == 0 && !mbar_wait(&k_full[sn], ((kv_it + 1) / NST) & 1u, abort_flag)) { ok = false; break; }
               tc_fence_after_sync();
-              issue_s(w, qb, sn);              // next scores first: the softmax of tile j+1 overlaps P V of tile j
+              issue_s(w, qb, sn);
             }
             if (w == 0 && !mbar_wait(&v_full[s], (kv_it / NST) & 1u, abort_flag)) { ok = false; break; }
             tc_fence_after_sync();
             issue_pv(w, s, j != 0);
+            if (last && has_next && w < un.n_q) {
+              // the unit's output is waiting for this P V, so it went first; now the first scores of the next unit
+              if (!next_q_ready) {
+                if (!mbar_wait(&q_full[qb ^ 1], ((u_cnt + 1) >> 1) & 1u, abort_flag)) { ok = false; break; }
+                next_q_ready = true;
+              }
+              if (w == 0 && !mbar_wait(&k_full[sn], ((kv_it + 1) / NST) & 1u, abort_flag)) { ok = false; break; }
+              tc_fence_after_sync();
+              issue_s(w, qb ^ 1, sn);
+              pre_issued[w] = true;
+            }
           }
           if (ok) umma_commit(&kv_empty[s]);   // K(j) and V(j) are free once everything issued so far completes
         }
@@ -317,13 +350,19 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_tc_kernel(const __grid_con
     uint32_t n = 0;                                // tiles processed by this warpgroup
     bool ok = true;
 
+    UnitInfo u_next = decode_unit(p, min(static_cast<int>(blockIdx.x), p.total_units - 1));
     for (int unit = blockIdx.x; unit < p.total_units && ok; unit += gridDim.x) {
-      const UnitInfo u = decode_unit(p, unit);
+      const UnitInfo u = u_next;
+      ATTN_STAMP_PREV(10);
+      // decode the following unit now, while this warp would otherwise wait for the first scores
+      if (unit + static_cast<int>(gridDim.x) < p.total_units) u_next = decode_unit(p, unit + gridDim.x);
       if (w >= u.n_q) continue;
       float m_used = -INFINITY, l = 0.f;
       for (int j = 0; j < u.n_kv; ++j, ++n) {
+        ATTN_STAMP(0);
         if (!mbar_wait(&s_full[w], n & 1u, abort_flag)) { ok = false; break; }
         tc_fence_after_sync();
+        ATTN_STAMP(1);
         const int valid = min(kTcTile, u.S - j * kTcTile);     // keys of this tile that belong to the item
         // the whole score row (128 fp32) in registers: four loads, one wait
         uint32_t sr[128];
@@ -333,6 +372,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_tc_kernel(const __grid_con
         tmem_ld_32x32_at<64>(s_addr, sr);
         tmem_ld_32x32_at<96>(s_addr, sr);
         tmem_ld_wait();
+        ATTN_STAMP(2);
         if (valid < kTcTile) {                                  // last tile of the item: keys past its end
 #pragma unroll
           for (int i = 0; i < 128; ++i) if (i >= valid) sr[i] = 0xff800000u;   // -inf
@@ -344,6 +384,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_tc_kernel(const __grid_con
           mx1 = fmax3(mx1, __uint_as_float(sr[i + 2]), __uint_as_float(sr[i + 3]));
         }
         const float mx = fmaxf(mx0, mx1);
+        ATTN_STAMP(3);
         // reference maximum: moves only when the row maximum grew by more than the threshold
         float corr = 1.0f;
         bool rescale = false;
@@ -386,7 +427,9 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_tc_kernel(const __grid_con
         }
         // S has been read: the issuer may overwrite it with the next tile's scores once p_ready fires.
         // The previous P V must be complete before P is overwritten or O is touched.
+        ATTN_STAMP(4);
         if (n > 0 && !mbar_wait(&pv_done[w], (n - 1) & 1u, abort_flag)) { ok = false; break; }
+        ATTN_STAMP(5);
         tc_fence_after_sync();
         if (__any_sync(0xffffffffu, rescale)) {
 #pragma unroll 1
@@ -412,34 +455,39 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_tc_kernel(const __grid_con
         tc_fence_before_sync();
         __syncwarp();
         if (lane == 0) mbar_arrive(&p_ready[w]);
+        ATTN_STAMP(6);
       }
       if (!ok) break;
       // epilogue: O / l -> bf16
       if (!mbar_wait(&pv_done[w], (n - 1) & 1u, abort_flag)) { ok = false; break; }
       tc_fence_after_sync();
+      ATTN_STAMP_PREV(7);
       const float inv = 1.0f / l;
       const int qrow = u.q0 + w * kTcTile + row;
       bf16* orow = p.out + (u.row0 + qrow) * p.ldo + u.head * HD;
-#pragma unroll 1
-      for (int c = 0; c < HD / 16; ++c) {
-        uint32_t o[16];
-        __syncwarp();
-        tmem_ld_32x16(o_addr + c * 16, o);
-        tmem_ld_wait();
-        if (qrow < u.S) {
-          uint4 v0 = make_uint4(pack_bf16x2(__uint_as_float(o[0]) * inv, __uint_as_float(o[1]) * inv),
-                                pack_bf16x2(__uint_as_float(o[2]) * inv, __uint_as_float(o[3]) * inv),
-                                pack_bf16x2(__uint_as_float(o[4]) * inv, __uint_as_float(o[5]) * inv),
-                                pack_bf16x2(__uint_as_float(o[6]) * inv, __uint_as_float(o[7]) * inv));
-          uint4 v1 = make_uint4(pack_bf16x2(__uint_as_float(o[8]) * inv, __uint_as_float(o[9]) * inv),
-                                pack_bf16x2(__uint_as_float(o[10]) * inv, __uint_as_float(o[11]) * inv),
-                                pack_bf16x2(__uint_as_float(o[12]) * inv, __uint_as_float(o[13]) * inv),
-                                pack_bf16x2(__uint_as_float(o[14]) * inv, __uint_as_float(o[15]) * inv));
+      uint32_t o[HD / 16][16];
+      __syncwarp();
+#pragma unroll
+      for (int c = 0; c < HD / 16; ++c) tmem_ld_32x16(o_addr + c * 16, o[c]);
+      tmem_ld_wait();
+      ATTN_STAMP_PREV(8);
+      if (qrow < u.S) {
+#pragma unroll
+        for (int c = 0; c < HD / 16; ++c) {
+          uint4 v0 = make_uint4(pack_bf16x2(__uint_as_float(o[c][0]) * inv, __uint_as_float(o[c][1]) * inv),
+                                pack_bf16x2(__uint_as_float(o[c][2]) * inv, __uint_as_float(o[c][3]) * inv),
+                                pack_bf16x2(__uint_as_float(o[c][4]) * inv, __uint_as_float(o[c][5]) * inv),
+                                pack_bf16x2(__uint_as_float(o[c][6]) * inv, __uint_as_float(o[c][7]) * inv));
+          uint4 v1 = make_uint4(pack_bf16x2(__uint_as_float(o[c][8]) * inv, __uint_as_float(o[c][9]) * inv),
+                                pack_bf16x2(__uint_as_float(o[c][10]) * inv, __uint_as_float(o[c][11]) * inv),
+                                pack_bf16x2(__uint_as_float(o[c][12]) * inv, __uint_as_float(o[c][13]) * inv),
+                                pack_bf16x2(__uint_as_float(o[c][14]) * inv, __uint_as_float(o[c][15]) * inv));
           uint4* dst = reinterpret_cast<uint4*>(orow + c * 16);
           dst[0] = v0;
           dst[1] = v1;
         }
       }
+      ATTN_STAMP_PREV(9);
       // the O reads above must complete before this warpgroup's next p_ready lets P V overwrite O
       tc_fence_before_sync();
     }

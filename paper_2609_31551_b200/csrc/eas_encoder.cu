@@ -1045,3 +1045,9 @@ extern "C" eas_status eas_kernel_attention(const void* qkv, void* out, const int
   return launch_attention(static_cast<const bf16*>(qkv), static_cast<bf16*>(out), cu, n_items, n_heads, head_dim, budget,
                           static_cast<cudaStream_t>(stream), impl, status_dev);
 }
+
+#ifdef EAS_ATTN_PROFILE
+extern "C" int eas_debug_attn_stamps(unsigned long long* host_out /* [2*64*12] */) {
+  return cudaMemcpyFromSymbol(host_out, eas::g_attn_dbg, sizeof(unsigned long long) * 2 * 64 * 12) == cudaSuccess ? 0 : 1;
+}
+#endif
