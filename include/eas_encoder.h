@@ -163,8 +163,9 @@ eas_status eas_encoder_status(eas_encoder* enc, void* stream);
 /* Number of kernel launches the last eas_encode_microbatch enqueued. */
 int32_t eas_encoder_last_launch_count(const eas_encoder* enc);
 
-/* Selects the attention kernel: 0 = default (tcgen05 / TMEM); 1 = register-tile (mma.sync) kernel, kept as a
- * cross-check for testing. */
+/* Selects the attention kernel: 0 = default (tcgen05, probabilities kept in tensor memory); 1 = register-tile
+ * (mma.sync) kernel; 2 = tcgen05 with the probabilities staged in shared memory.  1 and 2 are cross-checks for
+ * testing. */
 eas_status eas_encoder_set_attention_impl(eas_encoder* enc, int32_t impl);
 
 /* Per-kernel timing for profiling (off by default; adds one event record per launch).  Kernel classes: */

@@ -38,19 +38,39 @@ struct AttnTcParams {
   uint32_t* status;
 };
 
-template <int HD>
+// PT: the probabilities P live in tensor memory (the A operand of P V is read from there); otherwise they are
+// staged in shared memory.  With PT the 64 KB of P staging become extra K/V stages.
+template <int HD, bool PT>
 struct AttnTcSmem {
   static constexpr int HI = HD - 64;                       // 0 or 16 extra columns
   static constexpr int kLoBytes = kTcTile * 128;           // 128 rows x 64 bf16
   static constexpr int kHiBytes = kTcTile * HI * 2;        // 128 rows x 16 bf16
   static constexpr int kTileBytes = kLoBytes + kHiBytes;   // one Q, K or V tile
-  static constexpr int kStages = HD == 64 ? 3 : 2;
+  static constexpr int kStages = PT ? (HD == 64 ? 5 : 3) : (HD == 64 ? 3 : 2);
   static constexpr int kQOff = 0;                          // [2 buffers][2 tiles]
   static constexpr int kKvOff = kQOff + 4 * kTileBytes;    // [stages][K, V]
-  static constexpr int kPOff = kKvOff + kStages * 2 * kTileBytes;   // [2 tiles][2 k-blocks of 16 KB]
-  static constexpr int kBarOff = kPOff + 2 * 32768;
+  static constexpr int kPOff = kKvOff + kStages * 2 * kTileBytes;   // [2 tiles][2 k-blocks of 16 KB] (shared-memory P only)
+  static constexpr int kBarOff = kPOff + (PT ? 0 : 2 * 32768);
   static constexpr int kBytes = kBarOff + 512 + 1024;      // barriers + alignment slack
+  static_assert(kBytes <= 232448, "exceeds the shared memory of an SM");
+  // TMEM columns: S_A [0,128) S_B [128,256) O_A [256,256+HD) O_B [256+HD', ...).  P in tensor memory: head_dim 64 has
+  // room for dedicated columns; head_dim 80 re-uses the first 64 columns of S (dead once the row sits in registers),
+  // which obliges the issuer to run P V before the next S.
+  static constexpr int kOCol0 = 256, kOStride = HD == 64 ? 64 : 128;
+  static constexpr bool kPAliasesS = PT && HD != 64;
+  static constexpr int kPCol0 = kPAliasesS ? 0 : 384, kPStride = kPAliasesS ? 128 : 64;
 };
+__device__ __forceinline__ void tmem_st_32x32_from(uint32_t taddr, const uint32_t* r) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+      "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
+      ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+        "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]),
+        "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]),
+        "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+      : "memory");
+}
 
 __device__ __forceinline__ void tmem_ld_32x16(uint32_t taddr, uint32_t (&r)[16]) {
   asm volatile(
@@ -151,9 +171,9 @@ __device__ __forceinline__ UnitInfo decode_unit(const AttnTcParams& p, int unit)
   return u;
 }
 
-template <int HD>
+template <int HD, bool PT>
 __global__ void __launch_bounds__(kTcThreads, 1) attn_tc_kernel(const __grid_constant__ AttnTcParams p) {
-  using L = AttnTcSmem<HD>;
+  using L = AttnTcSmem<HD, PT>;
   constexpr int HI = L::HI;
   constexpr int NST = L::kStages;
   extern __shared__ uint8_t smem_raw_attn[];
@@ -193,7 +213,6 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_tc_kernel(const __grid_con
   const uint32_t tmem_base = *tmem_slot;
   pdl_launch_dependents();
   pdl_wait();
-  // TMEM columns: S_A [0,128)  S_B [128,256)  O_A [256,256+HD)  O_B [384,384+HD)
 
   auto q_tile = [&](int buf, int t) { return smem + L::kQOff + (buf * 2 + t) * L::kTileBytes; };
   auto k_tile = [&](int s) { return smem + L::kKvOff + (s * 2) * L::kTileBytes; };
@@ -263,17 +282,27 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_tc_kernel(const __grid_con
         ++n_tiles[w];
       };
       auto issue_pv = [&](int w, int s, bool accumulate) {
-        const uint32_t pa = smem_u32(p_tile(w));
         const uint32_t va = smem_u32(v_tile(s));
-        const uint32_t d = tmem_base + 256 + w * 128;
+        const uint32_t d = tmem_base + L::kOCol0 + w * L::kOStride;
 #pragma unroll
         for (int ks = 0; ks < 8; ++ks) {       // 16 keys per step
-          const uint64_t ad = make_smem_desc(pa + (ks >> 2) * 16384 + (ks & 3) * 32, 16, 1024, kSwizzle128B);
           const uint64_t bd = make_smem_desc(va + ks * 2048, 1024, 1024, kSwizzle128B);
-          umma_bf16_ss(d, ad, bd, idesc_o_lo, (accumulate || ks != 0) ? 1u : 0u);
-          if (HI) {
-            const uint64_t bh = make_smem_desc(va + L::kLoBytes + ks * 512, 256, 256, kSwizzle32B);
-            umma_bf16_ss(d + 64, ad, bh, idesc_o_hi, (accumulate || ks != 0) ? 1u : 0u);
+          const uint32_t acc = (accumulate || ks != 0) ? 1u : 0u;
+          if (PT) {
+            const uint32_t pt = tmem_base + L::kPCol0 + w * L::kPStride + ks * 8;   // 16 bf16 = 8 columns
+            umma_bf16_ts(d, pt, bd, idesc_o_lo, acc);
+            if (HI) {
+              const uint64_t bh = make_smem_desc(va + L::kLoBytes + ks * 512, 256, 256, kSwizzle32B);
+              umma_bf16_ts(d + 64, pt, bh, idesc_o_hi, acc);
+            }
+          } else {
+            const uint32_t pa = smem_u32(p_tile(w));
+            const uint64_t ad = make_smem_desc(pa + (ks >> 2) * 16384 + (ks & 3) * 32, 16, 1024, kSwizzle128B);
+            umma_bf16_ss(d, ad, bd, idesc_o_lo, acc);
+            if (HI) {
+              const uint64_t bh = make_smem_desc(va + L::kLoBytes + ks * 512, 256, 256, kSwizzle32B);
+              umma_bf16_ss(d + 64, ad, bh, idesc_o_hi, acc);
+            }
           }
         }
         umma_commit(&pv_done[w]);
@@ -309,7 +338,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_tc_kernel(const __grid_con
             tc_fence_after_sync();
             // next scores first (the softmax of the next tile overlaps P V of this one); after the unit's last
             // tile the next scores are the first tile of the NEXT unit, so the pipeline never drains
-            if (!last) {
+            // next scores before P V, so that the next softmax overlaps it -- unless P re-uses S's columns
+            if (!last && !L::kPAliasesS) {
               if (w == 0 && !mbar_wait(&k_full[sn], ((kv_it + 1) / NST) & 1u, abort_flag)) { ok = false; break; }
               tc_fence_after_sync();
               issue_s(w, qb, sn);
@@ -317,6 +347,11 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_tc_kernel(const __grid_con
             if (w == 0 && !mbar_wait(&v_full[s], (kv_it / NST) & 1u, abort_flag)) { ok = false; break; }
             tc_fence_after_sync();
             issue_pv(w, s, j != 0);
+            if (!last && L::kPAliasesS) {
+              if (w == 0 && !mbar_wait(&k_full[sn], ((kv_it + 1) / NST) & 1u, abort_flag)) { ok = false; break; }
+              tc_fence_after_sync();
+              issue_s(w, qb, sn);
+            }
             if (last && has_next && w < un.n_q) {
               // the unit's output is waiting for this P V, so it went first; now the first scores of the next unit
               if (!next_q_ready) {
@@ -344,7 +379,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_tc_kernel(const __grid_con
     const int row = quarter * 32 + lane;           // query row inside the tile == TMEM lane
     const uint32_t lane_addr = static_cast<uint32_t>(quarter * 32) << 16;
     const uint32_t s_addr = tmem_base + lane_addr + w * 128;
-    const uint32_t o_addr = tmem_base + lane_addr + 256 + w * 128;
+    const uint32_t o_addr = tmem_base + lane_addr + L::kOCol0 + w * L::kOStride;
+    const uint32_t p_addr = tmem_base + lane_addr + L::kPCol0 + w * L::kPStride;
     uint8_t* p_row = p_tile(w) + row * 128;
     const int sw = row & 7;
     uint32_t n = 0;                                // tiles processed by this warpgroup
@@ -444,14 +480,22 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_tc_kernel(const __grid_con
           }
           tmem_st_wait();
         }
-        // P row: 2 k-blocks of 64 keys, each row 128 bytes, 16-byte chunks XOR-swizzled by (row & 7)
+        if (PT) {
+          // P row into tensor memory: 128 bf16 = 64 columns of this thread's lane
+          __syncwarp();
+          tmem_st_32x32_from(p_addr, pk);
+          tmem_st_32x32_from(p_addr + 32, pk + 32);
+          tmem_st_wait();
+        } else {
+          // P row: 2 k-blocks of 64 keys, each row 128 bytes, 16-byte chunks XOR-swizzled by (row & 7)
 #pragma unroll
-        for (int cc = 0; cc < 16; ++cc) {
-          const int kblk = cc >> 3, ch = cc & 7;
-          uint4 v = make_uint4(pk[cc * 4], pk[cc * 4 + 1], pk[cc * 4 + 2], pk[cc * 4 + 3]);
-          *reinterpret_cast<uint4*>(p_row + kblk * 16384 + ((ch ^ sw) << 4)) = v;
+          for (int cc = 0; cc < 16; ++cc) {
+            const int kblk = cc >> 3, ch = cc & 7;
+            uint4 v = make_uint4(pk[cc * 4], pk[cc * 4 + 1], pk[cc * 4 + 2], pk[cc * 4 + 3]);
+            *reinterpret_cast<uint4*>(p_row + kblk * 16384 + ((ch ^ sw) << 4)) = v;
+          }
+          fence_proxy_async_smem();
         }
-        fence_proxy_async_smem();
         tc_fence_before_sync();
         __syncwarp();
         if (lane == 0) mbar_arrive(&p_ready[w]);

@@ -418,7 +418,7 @@ extern "C" eas_status eas_encoder_create(const eas_arch_config* arch, const eas_
 extern "C" void eas_encoder_destroy(eas_encoder* enc) { delete enc; }
 
 extern "C" eas_status eas_encoder_set_attention_impl(eas_encoder* enc, int32_t impl) {
-  if (enc == nullptr || impl < 0 || impl > 1) return fail(EAS_ERR_INVALID_ARG, "bad attention impl");
+  if (enc == nullptr || impl < 0 || impl > 2) return fail(EAS_ERR_INVALID_ARG, "bad attention impl");
   enc->attn_impl = impl;
   return EAS_OK;
 }
@@ -638,6 +638,7 @@ static eas_status launch_attention_mma(const bf16* qkv, bf16* out, const int32_t
   return fail(EAS_ERR_UNSUPPORTED, "head_dim %d", hd);
 }
 
+template <bool PT>
 static eas_status launch_attention_tc(const bf16* qkv, bf16* out, const int32_t* cu, int n_items, int H, int hd, int budget,
                                       cudaStream_t stream, uint32_t* status) {
   AttnTcParams ap{};
@@ -660,19 +661,20 @@ static eas_status launch_attention_tc(const bf16* qkv, bf16* out, const int32_t*
   const int grid = std::min(budget, ap.total_units);
   static bool attr_set = false;
   if (!attr_set) {
-    CUDA_TRY(cudaFuncSetAttribute(attn_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttnTcSmem<64>::kBytes));
-    CUDA_TRY(cudaFuncSetAttribute(attn_tc_kernel<80>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttnTcSmem<80>::kBytes));
+    CUDA_TRY(cudaFuncSetAttribute(attn_tc_kernel<64, PT>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttnTcSmem<64, PT>::kBytes));
+    CUDA_TRY(cudaFuncSetAttribute(attn_tc_kernel<80, PT>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttnTcSmem<80, PT>::kBytes));
     attr_set = true;
   }
-  if (hd == 64) return launch_kernel(attn_tc_kernel<64>, grid, kTcThreads, AttnTcSmem<64>::kBytes, stream, ap);
-  if (hd == 80) return launch_kernel(attn_tc_kernel<80>, grid, kTcThreads, AttnTcSmem<80>::kBytes, stream, ap);
+  if (hd == 64) return launch_kernel(attn_tc_kernel<64, PT>, grid, kTcThreads, AttnTcSmem<64, PT>::kBytes, stream, ap);
+  if (hd == 80) return launch_kernel(attn_tc_kernel<80, PT>, grid, kTcThreads, AttnTcSmem<80, PT>::kBytes, stream, ap);
   return fail(EAS_ERR_UNSUPPORTED, "head_dim %d", hd);
 }
 
 static eas_status launch_attention(const bf16* qkv, bf16* out, const int32_t* cu, int n_items, int H, int hd, int budget,
                                    cudaStream_t stream, int impl, uint32_t* status) {
   if (impl == 1) return launch_attention_mma(qkv, out, cu, n_items, H, hd, budget, stream);
-  return launch_attention_tc(qkv, out, cu, n_items, H, hd, budget, stream, status);
+  if (impl == 2) return launch_attention_tc<false>(qkv, out, cu, n_items, H, hd, budget, stream, status);
+  return launch_attention_tc<true>(qkv, out, cu, n_items, H, hd, budget, stream, status);
 }
 
 // ------------------------------------------------------------------------------------ the forward pass

@@ -100,7 +100,7 @@ def test_norm(d, kind):
 
 @pytest.mark.parametrize("hd,H", [(64, 3), (80, 2)])
 @pytest.mark.parametrize("lens", [[5], [128], [129, 1, 64, 577], [200, 1000]])
-@pytest.mark.parametrize("impl", [0, 1])
+@pytest.mark.parametrize("impl", [0, 1, 2])
 def test_attention_block_diagonal(hd, H, lens, impl):
     import paper_2609_31551_b200 as P
     rng = np.random.Generator(np.random.PCG64(hd + len(lens) + sum(lens)))
