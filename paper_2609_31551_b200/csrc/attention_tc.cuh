@@ -27,6 +27,7 @@ constexpr float kRescaleThreshold = 8.0f;
 struct AttnTcParams {
   CUtensorMap map_lo;   // qkv [T, 3d], box {64 columns, 128 rows}, 128-byte swizzle
   CUtensorMap map_hi;   // box {16 columns, 128 rows}, 32-byte swizzle (head_dim 80: columns 64..79)
+  CUtensorMap map_out;  // out [T, d], box {64 columns, 32 rows}, 128-byte swizzle (store of a warp's 32 output rows)
   bf16* out;
   long long ldo;
   int d_model, n_heads;
@@ -46,11 +47,13 @@ struct AttnTcSmem {
   static constexpr int kLoBytes = kTcTile * 128;           // 128 rows x 64 bf16
   static constexpr int kHiBytes = kTcTile * HI * 2;        // 128 rows x 16 bf16
   static constexpr int kTileBytes = kLoBytes + kHiBytes;   // one Q, K or V tile
-  static constexpr int kStages = PT ? (HD == 64 ? 5 : 3) : (HD == 64 ? 3 : 2);
+  static constexpr bool kStagedOut = PT && HD == 64;       // output rows leave through shared memory and TMA stores
+  static constexpr int kStages = PT ? (HD == 64 ? 4 : 3) : (HD == 64 ? 3 : 2);
   static constexpr int kQOff = 0;                          // [2 buffers][2 tiles]
   static constexpr int kKvOff = kQOff + 4 * kTileBytes;    // [stages][K, V]
   static constexpr int kPOff = kKvOff + kStages * 2 * kTileBytes;   // [2 tiles][2 k-blocks of 16 KB] (shared-memory P only)
-  static constexpr int kBarOff = kPOff + (PT ? 0 : 2 * 32768);
+  static constexpr int kOutOff = kPOff + (PT ? 0 : 2 * 32768);      // [8 softmax warps][32 rows x 128 bytes]
+  static constexpr int kBarOff = kOutOff + (kStagedOut ? 8 * 4096 : 0);
   static constexpr int kBytes = kBarOff + 512 + 1024;      // barriers + alignment slack
   static_assert(kBytes <= 232448, "exceeds the shared memory of an SM");
   // TMEM columns: S_A [0,128) S_B [128,256) O_A [256,256+HD) O_B [256+HD', ...).  P in tensor memory: head_dim 64 has
@@ -153,12 +156,12 @@ struct UnitInfo {
   int head, q0, S, n_kv, n_q;
   long long row0;
 };
-__device__ __forceinline__ UnitInfo decode_unit(const AttnTcParams& p, int unit) {
-  int lo = 0, hi = p.n_items - 1;
-  while (lo < hi) {
-    const int mid = (lo + hi + 1) >> 1;
-    if (p.unit_prefix[mid] <= unit) lo = mid; else hi = mid - 1;
-  }
+// `cursor` is the caller's item index of its previous unit: units are visited in increasing order, so the item is
+// found by stepping forward (usually zero or one step) instead of searching.
+__device__ __forceinline__ UnitInfo decode_unit(const AttnTcParams& p, int unit, int& cursor) {
+  int lo = cursor;
+  while (lo + 1 < p.n_items && p.unit_prefix[lo + 1] <= unit) ++lo;
+  cursor = lo;
   UnitInfo u;
   u.S = p.item_len[lo];
   u.row0 = p.item_start[lo];
@@ -225,8 +228,9 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_tc_kernel(const __grid_con
     if (lane == 0) {
       uint32_t kv_it = 0, u_cnt = 0;
       bool ok = true;
+      int cursor = 0;
       for (int unit = blockIdx.x; unit < p.total_units && ok; unit += gridDim.x, ++u_cnt) {
-        const UnitInfo u = decode_unit(p, unit);
+        const UnitInfo u = decode_unit(p, unit, cursor);
         const int qb = u_cnt & 1;
         if (!mbar_wait(&q_empty[qb], ((u_cnt >> 1) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
         mbar_expect_tx(&q_full[qb], u.n_q * L::kTileBytes);
@@ -310,12 +314,13 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_tc_kernel(const __grid_con
       };
 
       bool pre_issued[2] = {false, false};       // S(w, 0) of this unit was already issued at the end of the previous one
+      int cursor = 0;
+      UnitInfo un = decode_unit(p, min(static_cast<int>(blockIdx.x), p.total_units - 1), cursor);
       for (int unit = blockIdx.x; unit < p.total_units && ok; unit += gridDim.x, ++u_cnt) {
-        const UnitInfo u = decode_unit(p, unit);
+        const UnitInfo u = un;
         const int qb = u_cnt & 1;
         const bool has_next = unit + static_cast<int>(gridDim.x) < p.total_units;
-        UnitInfo un = u;
-        if (has_next) un = decode_unit(p, unit + gridDim.x);
+        if (has_next) un = decode_unit(p, unit + gridDim.x, cursor);
         if (!mbar_wait(&q_full[qb], (u_cnt >> 1) & 1u, abort_flag)) { ok = false; break; }
         {
           const int s = kv_it % NST;
@@ -386,13 +391,73 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_tc_kernel(const __grid_con
     uint32_t n = 0;                                // tiles processed by this warpgroup
     bool ok = true;
 
-    UnitInfo u_next = decode_unit(p, min(static_cast<int>(blockIdx.x), p.total_units - 1));
+    // The output of a unit is written while the NEXT unit's first tile is in flight: by then its last P V has
+    // long finished, so the warpgroup never waits for it.
+    bool pend = false;
+    int pend_q0 = 0, pend_head = 0, pend_S = 0;
+    long long pend_row0 = 0;
+    float pend_l = 1.f;
+    uint32_t pend_n = 0;
+    uint8_t* out_stage = smem + L::kOutOff + (warp - 4) * 4096;
+    auto flush_output = [&]() -> bool {
+      if (!mbar_wait(&pv_done[w], pend_n & 1u, abort_flag)) return false;
+      tc_fence_after_sync();
+      ATTN_STAMP_PREV(7);
+      const float inv = 1.0f / pend_l;
+      const int warp_row0 = pend_q0 + w * kTcTile + quarter * 32;      // first query row of this warp within the item
+      const int qrow = warp_row0 + lane;
+      uint32_t o[HD / 16][16];
+      __syncwarp();
+#pragma unroll
+      for (int c = 0; c < HD / 16; ++c) tmem_ld_32x16(o_addr + c * 16, o[c]);
+      tmem_ld_wait();
+      ATTN_STAMP_PREV(8);
+      uint32_t pkd[HD / 2];
+#pragma unroll
+      for (int c = 0; c < HD / 16; ++c)
+#pragma unroll
+        for (int i = 0; i < 8; ++i)
+          pkd[c * 8 + i] = pack_bf16x2(__uint_as_float(o[c][2 * i]) * inv, __uint_as_float(o[c][2 * i + 1]) * inv);
+      if (L::kStagedOut && warp_row0 + 32 <= pend_S) {
+        // all 32 rows of this warp belong to the item: swizzled staging, one TMA store
+        if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+        __syncwarp();
+        uint8_t* srow = out_stage + lane * 128;
+#pragma unroll
+        for (int q = 0; q < 8; ++q)
+          *reinterpret_cast<uint4*>(srow + ((q ^ (lane & 7)) << 4)) = make_uint4(pkd[4 * q], pkd[4 * q + 1], pkd[4 * q + 2], pkd[4 * q + 3]);
+        fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0) {
+          asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
+                       ::"l"(reinterpret_cast<uint64_t>(&p.map_out)), "r"(smem_u32(out_stage)), "r"(pend_head * HD),
+                         "r"(static_cast<int>(pend_row0) + warp_row0) : "memory");
+          asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+        }
+      } else if (qrow < pend_S) {
+        // the warp straddles the item's end (or this head size has no staged path): per-row stores
+        uint4* dst = reinterpret_cast<uint4*>(p.out + (pend_row0 + qrow) * p.ldo + pend_head * HD);
+#pragma unroll
+        for (int q = 0; q < HD / 8; ++q) dst[q] = make_uint4(pkd[4 * q], pkd[4 * q + 1], pkd[4 * q + 2], pkd[4 * q + 3]);
+      }
+      ATTN_STAMP_PREV(9);
+      // the O reads above are complete before this warpgroup's next p_ready lets P V overwrite O
+      tc_fence_before_sync();
+      pend = false;
+      return true;
+    };
+
+    int cursor = 0;
+    UnitInfo u_next = decode_unit(p, min(static_cast<int>(blockIdx.x), p.total_units - 1), cursor);
     for (int unit = blockIdx.x; unit < p.total_units && ok; unit += gridDim.x) {
       const UnitInfo u = u_next;
       ATTN_STAMP_PREV(10);
-      // decode the following unit now, while this warp would otherwise wait for the first scores
-      if (unit + static_cast<int>(gridDim.x) < p.total_units) u_next = decode_unit(p, unit + gridDim.x);
-      if (w >= u.n_q) continue;
+      const bool has_next = unit + static_cast<int>(gridDim.x) < p.total_units;
+      if (w >= u.n_q) {                             // this warpgroup has no tile in the unit
+        if (has_next) u_next = decode_unit(p, unit + gridDim.x, cursor);
+        if (pend && !flush_output()) { ok = false; break; }
+        continue;
+      }
       float m_used = -INFINITY, l = 0.f;
       for (int j = 0; j < u.n_kv; ++j, ++n) {
         ATTN_STAMP(0);
@@ -464,6 +529,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_tc_kernel(const __grid_con
         // S has been read: the issuer may overwrite it with the next tile's scores once p_ready fires.
         // The previous P V must be complete before P is overwritten or O is touched.
         ATTN_STAMP(4);
+        if (j == 0 && pend && !flush_output()) { ok = false; break; }
         if (n > 0 && !mbar_wait(&pv_done[w], (n - 1) & 1u, abort_flag)) { ok = false; break; }
         ATTN_STAMP(5);
         tc_fence_after_sync();
@@ -500,41 +566,15 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_tc_kernel(const __grid_con
         __syncwarp();
         if (lane == 0) mbar_arrive(&p_ready[w]);
         ATTN_STAMP(6);
+        // decode the following unit here: the warp now waits for the issuer anyway
+        if (j == 0 && has_next) u_next = decode_unit(p, unit + gridDim.x, cursor);
       }
       if (!ok) break;
-      // epilogue: O / l -> bf16
-      if (!mbar_wait(&pv_done[w], (n - 1) & 1u, abort_flag)) { ok = false; break; }
-      tc_fence_after_sync();
-      ATTN_STAMP_PREV(7);
-      const float inv = 1.0f / l;
-      const int qrow = u.q0 + w * kTcTile + row;
-      bf16* orow = p.out + (u.row0 + qrow) * p.ldo + u.head * HD;
-      uint32_t o[HD / 16][16];
-      __syncwarp();
-#pragma unroll
-      for (int c = 0; c < HD / 16; ++c) tmem_ld_32x16(o_addr + c * 16, o[c]);
-      tmem_ld_wait();
-      ATTN_STAMP_PREV(8);
-      if (qrow < u.S) {
-#pragma unroll
-        for (int c = 0; c < HD / 16; ++c) {
-          uint4 v0 = make_uint4(pack_bf16x2(__uint_as_float(o[c][0]) * inv, __uint_as_float(o[c][1]) * inv),
-                                pack_bf16x2(__uint_as_float(o[c][2]) * inv, __uint_as_float(o[c][3]) * inv),
-                                pack_bf16x2(__uint_as_float(o[c][4]) * inv, __uint_as_float(o[c][5]) * inv),
-                                pack_bf16x2(__uint_as_float(o[c][6]) * inv, __uint_as_float(o[c][7]) * inv));
-          uint4 v1 = make_uint4(pack_bf16x2(__uint_as_float(o[c][8]) * inv, __uint_as_float(o[c][9]) * inv),
-                                pack_bf16x2(__uint_as_float(o[c][10]) * inv, __uint_as_float(o[c][11]) * inv),
-                                pack_bf16x2(__uint_as_float(o[c][12]) * inv, __uint_as_float(o[c][13]) * inv),
-                                pack_bf16x2(__uint_as_float(o[c][14]) * inv, __uint_as_float(o[c][15]) * inv));
-          uint4* dst = reinterpret_cast<uint4*>(orow + c * 16);
-          dst[0] = v0;
-          dst[1] = v1;
-        }
-      }
-      ATTN_STAMP_PREV(9);
-      // the O reads above must complete before this warpgroup's next p_ready lets P V overwrite O
-      tc_fence_before_sync();
+      pend = true;                                  // written later, see flush_output
+      pend_q0 = u.q0; pend_head = u.head; pend_S = u.S; pend_row0 = u.row0; pend_l = l; pend_n = n - 1;
     }
+    if (ok && pend) flush_output();
+    if (L::kStagedOut && lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
   }
 
   tc_fence_before_sync();

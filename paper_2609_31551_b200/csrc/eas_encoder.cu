@@ -651,6 +651,10 @@ static eas_status launch_attention_tc(const bf16* qkv, bf16* out, const int32_t*
     EAS_TRY(make_tmap(&ap.map_lo, qkv, 2, dims, strides, box_lo, CU_TENSOR_MAP_SWIZZLE_128B));
     const uint32_t box_hi[2] = {16, kTcTile};
     EAS_TRY(make_tmap(&ap.map_hi, qkv, 2, dims, strides, box_hi, CU_TENSOR_MAP_SWIZZLE_32B));
+    const uint64_t odims[2] = {static_cast<uint64_t>(d), static_cast<uint64_t>(T)};
+    const uint64_t ostrides[1] = {static_cast<uint64_t>(d) * 2};
+    const uint32_t obox[2] = {64, 32};
+    EAS_TRY(make_tmap(&ap.map_out, out, 2, odims, ostrides, obox, CU_TENSOR_MAP_SWIZZLE_128B));
   }
   ap.out = out; ap.ldo = d; ap.d_model = d; ap.n_heads = H;
   ap.scale_log2 = static_cast<float>(1.4426950408889634 / std::sqrt(static_cast<double>(hd)));
