@@ -32,6 +32,12 @@ def test_library_exports_every_declared_symbol(lib):
         assert hasattr(lib, name), f"{name} is declared in include/eas_encoder.h but not exported"
     from paper_2609_31551_b200.binding import EXPORTED_SYMBOLS
     assert declared == set(EXPORTED_SYMBOLS)
+    header2 = open(os.path.join(ROOT, "include", "eas_serving.h")).read()
+    declared2 = set(re.findall(r"\b(eas_[a-z_0-9]+)\s*\(", header2))
+    from paper_2609_31551_b200.serving import SERVING_SYMBOLS
+    assert declared2 == set(SERVING_SYMBOLS)
+    for name in sorted(declared2):
+        assert hasattr(lib, name), f"{name} is declared in include/eas_serving.h but not exported"
 
 
 def test_arena_size_and_config_validation_run_on_the_host(lib):
