@@ -128,6 +128,30 @@ __device__ __forceinline__ uint64_t fadd2(uint64_t a, uint64_t b) {
   asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
   return d;
 }
+// 2^x for a pair of arguments on the FMA pipe instead of the special-function unit: x = n + f with n = rint(x)
+// (magic-number rounding), 2^f by a cubic fitted on [-0.5, 0.5] (relative error below 8e-5, far under the bf16
+// rounding of P), then n is added to the exponent field.  Arguments are clamped at -126 (result ~1e-38 instead of 0).
+#ifndef EAS_ATTN_POLY_OF_4
+#define EAS_ATTN_POLY_OF_4 1      // of every 4 pairs of probabilities, this many take the polynomial path
+#endif
+__device__ __forceinline__ void exp2_poly_pair(uint64_t x2, float& p0, float& p1) {
+  float x0, x1;
+  unpack2(x2, x0, x1);
+  x2 = pack2(fmaxf(x0, -126.0f), fmaxf(x1, -126.0f));
+  const uint64_t magic = pack2(12582912.0f, 12582912.0f);            // 1.5 * 2^23
+  const uint64_t nmagic = pack2(-12582912.0f, -12582912.0f);
+  const uint64_t t2 = fadd2(x2, magic);                              // low mantissa bits hold rint(x)
+  const uint64_t n2 = fadd2(t2, nmagic);
+  const uint64_t f2 = ffma2(n2, pack2(-1.0f, -1.0f), x2);            // f = x - n in [-0.5, 0.5]
+  uint64_t r2 = ffma2(pack2(0.05508868f, 0.05508868f), f2, pack2(0.24260405f, 0.24260405f));
+  r2 = ffma2(r2, f2, pack2(0.69327623f, 0.69327623f));
+  r2 = ffma2(r2, f2, pack2(0.99992895f, 0.99992895f));
+  float r0, r1, t0, t1;
+  unpack2(r2, r0, r1);
+  unpack2(t2, t0, t1);
+  p0 = __uint_as_float(__float_as_uint(r0) + (__float_as_uint(t0) << 23));
+  p1 = __uint_as_float(__float_as_uint(r1) + (__float_as_uint(t1) << 23));
+}
 __device__ __forceinline__ float fmax3(float a, float b, float c) {
   float d;
   asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
@@ -508,10 +532,15 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_tc_kernel(const __grid_con
 #pragma unroll
           for (int q = 0; q < 4; ++q) {
             const uint64_t t = ffma2(pack2(__uint_as_float(sr[2 * (i + q)]), __uint_as_float(sr[2 * (i + q) + 1])), scale2, nmb2);
-            float t0, t1;
-            unpack2(t, t0, t1);
-            const float p0 = fast_ex2(t0);
-            const float p1 = fast_ex2(t1);
+            float p0, p1;
+            if (q < EAS_ATTN_POLY_OF_4) {
+              exp2_poly_pair(t, p0, p1);
+            } else {
+              float t0, t1;
+              unpack2(t, t0, t1);
+              p0 = fast_ex2(t0);
+              p1 = fast_ex2(t1);
+            }
             const uint64_t pp = pack2(p0, p1);
             if (q == 0) acc0 = fadd2(acc0, pp);
             if (q == 1) acc1 = fadd2(acc1, pp);
