@@ -109,25 +109,6 @@ __device__ __forceinline__ void tmem_ld_32x32_at(uint32_t taddr, uint32_t (&r)[1
       : "r"(taddr + OFF)
       : "memory");
 }
-// packed fp32x2 arithmetic (two lanes per instruction on the FMA pipe)
-__device__ __forceinline__ uint64_t pack2(float lo, float hi) {
-  uint64_t d;
-  asm("mov.b64 %0, {%1, %2};" : "=l"(d) : "f"(lo), "f"(hi));
-  return d;
-}
-__device__ __forceinline__ void unpack2(uint64_t v, float& lo, float& hi) {
-  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
-}
-__device__ __forceinline__ uint64_t ffma2(uint64_t a, uint64_t b, uint64_t c) {
-  uint64_t d;
-  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
-  return d;
-}
-__device__ __forceinline__ uint64_t fadd2(uint64_t a, uint64_t b) {
-  uint64_t d;
-  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
-  return d;
-}
 // 2^x for a pair of arguments on the FMA pipe instead of the special-function unit: x = n + f with n = rint(x)
 // (magic-number rounding), 2^f by a cubic fitted on [-0.5, 0.5] (relative error below 8e-5, far under the bf16
 // rounding of P), then n is added to the exponent field.  Arguments are clamped at -126 (result ~1e-38 instead of 0).

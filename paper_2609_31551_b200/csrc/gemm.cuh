@@ -248,7 +248,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_kernel(const __grid_cons
           }
           if (ACT == ACT_GELU) {
 #pragma unroll
-            for (int i = 0; i < 32; ++i) v[i] = gelu_erf(v[i]);
+            for (int i = 0; i < 32; i += 2) gelu_erf_pair(v[i], v[i + 1]);
           }
         };
         auto staging_free = [&]() {       // the previous bulk store has finished READING the staging buffer

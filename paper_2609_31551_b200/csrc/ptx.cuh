@@ -254,6 +254,51 @@ __device__ __forceinline__ float gelu_erf(float x) {
   const float hx = 0.5f * x;
   return fmaf(hx, erf_fast(x * 0.70710678118654752f), hx);
 }
+// packed fp32x2 arithmetic (two lanes per instruction on the FMA pipe)
+__device__ __forceinline__ uint64_t pack2(float lo, float hi) {
+  uint64_t d;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(d) : "f"(lo), "f"(hi));
+  return d;
+}
+__device__ __forceinline__ void unpack2(uint64_t v, float& lo, float& hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t ffma2(uint64_t a, uint64_t b, uint64_t c) {
+  uint64_t d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ uint64_t fadd2(uint64_t a, uint64_t b) {
+  uint64_t d;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+__device__ __forceinline__ uint64_t fmul2(uint64_t a, uint64_t b) {
+  uint64_t d;
+  asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+// GELU (erf form, same rational-exponential erf as gelu_erf) on two values at once with packed fp32x2 arithmetic
+__device__ __forceinline__ void gelu_erf_pair(float& x0, float& x1) {
+  const uint64_t x2 = pack2(x0, x1);
+  const uint64_t az2 = pack2(fabsf(x0) * 0.70710678118654752f, fabsf(x1) * 0.70710678118654752f);
+  float d0, d1;
+  unpack2(ffma2(pack2(0.3275911f, 0.3275911f), az2, pack2(1.0f, 1.0f)), d0, d1);
+  const uint64_t t2 = pack2(fast_rcp(d0), fast_rcp(d1));
+  uint64_t p2 = ffma2(pack2(1.061405429f, 1.061405429f), t2, pack2(-1.453152027f, -1.453152027f));
+  p2 = ffma2(p2, t2, pack2(1.421413741f, 1.421413741f));
+  p2 = ffma2(p2, t2, pack2(-0.284496736f, -0.284496736f));
+  p2 = ffma2(p2, t2, pack2(0.254829592f, 0.254829592f));
+  p2 = fmul2(p2, t2);
+  float e0, e1;
+  unpack2(fmul2(fmul2(az2, az2), pack2(-1.4426950408889634f, -1.4426950408889634f)), e0, e1);
+  const uint64_t e2 = pack2(fast_ex2(e0), fast_ex2(e1));
+  float r0, r1;
+  unpack2(ffma2(fmul2(p2, pack2(-1.0f, -1.0f)), e2, pack2(1.0f, 1.0f)), r0, r1);   // erf(|z|) = 1 - p e
+  const uint64_t erf2 = pack2(copysignf(r0, x0), copysignf(r1, x1));
+  const uint64_t hx2 = fmul2(x2, pack2(0.5f, 0.5f));
+  unpack2(ffma2(hx2, erf2, hx2), x0, x1);
+}
 __device__ __forceinline__ float silu_f(float x) {
   return x * fast_rcp(1.0f + fast_ex2(-1.4426950408889634f * x));
 }
