@@ -83,6 +83,26 @@ int32_t eas_sm_table_build(const int32_t* sm_counts, int32_t n_levels, const int
  * (the value to pass as sm_budget), or -1 on a bad table. */
 int32_t eas_sm_table_lookup(const eas_sm_table* t, int32_t batch);
 
+/* ---- Section 3.1, Algorithm 1 lines 1-12, Eq. 3 and Eq. 4: Stage 1 of the configuration search ------------------- */
+
+/* One candidate allocation of workers to stages and what Stage 1 derives for it. */
+typedef struct {
+  int32_t n_encode, n_prefill, n_decode; /* workers per stage (inputs) */
+  int32_t n_local;                       /* co-resident local prefill workers on encode GPUs (input) */
+  double rho_e, rho_p, rho_d;            /* utilisations: (Lambda/n)/C; prefill: Lambda / (C_P (n_P + n_L alpha)) */
+  double score;                          /* max of the three */
+  int32_t b_max;                         /* ceil(Lambda / n_E): cap of the batch bound B for Stage 2 */
+  double s_star;                         /* n_P / (n_P + n_L alpha): centre of the offload-ratio window (+-0.2) */
+  int32_t kept;                          /* 1 if the allocation survives all three filters */
+} eas_has_candidate;
+
+/* Scores every candidate in place, discards score >= 1, prunes score > prune_factor x the minimum surviving score
+ * (1.2 in the paper), keeps the top_k best (3 in the paper; ties keep the earlier candidate).  c_e, c_p, c_d: profiled
+ * per-worker capacities in requests/s; alpha in [0,1]: memory share of a local prefill worker.  Returns the number
+ * kept, or -1 on a bad argument. */
+int32_t eas_has_stage1(eas_has_candidate* cand, int32_t n_candidates, double target_rate, double c_e, double c_p,
+                       double c_d, double alpha, double prune_factor, int32_t top_k);
+
 #ifdef __cplusplus
 }
 #endif

@@ -83,3 +83,20 @@ def sm_table_lookup(table, batch):
         if mb >= batch:
             return sm
     return table[-1][0]
+
+
+def has_stage1(cands, rate, c_e, c_p, c_d, alpha, prune=1.2, top_k=3):
+    """Algorithm 1, lines 1-12 (Eq. 3, Eq. 4).  cands: [(n_E, n_P, n_D, n_L)].  Returns (rows, kept indices) with
+    rows = (rho_E, rho_P, rho_D, score, B_max, s*)."""
+    rows = []
+    for nE, nP, nD, nL in cands:
+        pw = nP + nL * alpha
+        rE, rP, rD = (rate / nE) / c_e, (rate / (c_p * pw) if pw > 0 else math.inf), (rate / nD) / c_d
+        rows.append((rE, rP, rD, max(rE, rP, rD), math.ceil(rate / nE), (nP / pw if pw > 0 else 0.0)))
+    alive = [i for i, r in enumerate(rows) if r[3] < 1.0]
+    if not alive:
+        return rows, []
+    best = min(rows[i][3] for i in alive)
+    alive = [i for i in alive if rows[i][3] <= prune * best]
+    alive.sort(key=lambda i: rows[i][3])          # stable: ties keep the earlier candidate
+    return rows, sorted(alive[:top_k])

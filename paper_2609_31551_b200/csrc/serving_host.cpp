@@ -5,6 +5,8 @@
 #include <cmath>
 #include <limits>
 #include <new>
+#include <vector>
+#include <algorithm>
 
 // ------------------------------------------------------------------------------------ micro-batcher (Eq. 5)
 extern "C" double eas_poisson_gap_kappa(int32_t B, double p) {
@@ -136,4 +138,35 @@ extern "C" int32_t eas_sm_table_lookup(const eas_sm_table* t, int32_t batch) {
   for (int32_t l = 0; l < t->n_levels; ++l)
     if (t->max_batch[l] >= batch) return t->sm_count[l];
   return t->sm_count[t->n_levels - 1];
+}
+
+// ------------------------------------------------------------------------------------ HAS Stage 1 (Eq. 3, Eq. 4)
+extern "C" int32_t eas_has_stage1(eas_has_candidate* c, int32_t n, double rate, double c_e, double c_p, double c_d,
+                                  double alpha, double prune_factor, int32_t top_k) {
+  if (c == nullptr || n < 1 || !(rate > 0) || !(c_e > 0) || !(c_p > 0) || !(c_d > 0) || !(alpha >= 0 && alpha <= 1) ||
+      !(prune_factor >= 1) || top_k < 1)
+    return -1;
+  const double inf = std::numeric_limits<double>::infinity();
+  double best = inf;
+  for (int32_t i = 0; i < n; ++i) {
+    eas_has_candidate& a = c[i];
+    if (a.n_encode < 1 || a.n_prefill < 0 || a.n_decode < 1 || a.n_local < 0) return -1;
+    const double prefill_workers = a.n_prefill + a.n_local * alpha;
+    a.rho_e = (rate / a.n_encode) / c_e;
+    a.rho_p = prefill_workers > 0 ? rate / (c_p * prefill_workers) : inf;
+    a.rho_d = (rate / a.n_decode) / c_d;
+    a.score = std::max(a.rho_e, std::max(a.rho_p, a.rho_d));
+    a.b_max = static_cast<int32_t>(std::ceil(rate / a.n_encode));
+    a.s_star = prefill_workers > 0 ? a.n_prefill / prefill_workers : 0.0;
+    a.kept = a.score < 1.0 ? 1 : 0;                     // an overloaded stage rules the allocation out
+    if (a.kept) best = std::min(best, a.score);
+  }
+  std::vector<int32_t> order;
+  for (int32_t i = 0; i < n; ++i) {
+    if (c[i].kept && c[i].score > prune_factor * best) c[i].kept = 0;
+    if (c[i].kept) order.push_back(i);
+  }
+  std::stable_sort(order.begin(), order.end(), [&](int32_t x, int32_t y) { return c[x].score < c[y].score; });
+  for (size_t k = static_cast<size_t>(top_k); k < order.size(); ++k) c[order[k]].kept = 0;
+  return static_cast<int32_t>(std::min<size_t>(order.size(), static_cast<size_t>(top_k)));
 }

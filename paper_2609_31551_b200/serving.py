@@ -7,8 +7,14 @@ from .binding import load_library
 SERVING_SYMBOLS = [
     "eas_poisson_gap_kappa", "eas_batcher_create", "eas_batcher_destroy", "eas_batcher_gap", "eas_batcher_deadline",
     "eas_batcher_on_arrival", "eas_batcher_on_timer", "eas_router_init", "eas_router_init_from_double", "eas_router_next",
-    "eas_envelope_plan", "eas_sm_table_build", "eas_sm_table_lookup",
+    "eas_envelope_plan", "eas_sm_table_build", "eas_sm_table_lookup", "eas_has_stage1",
 ]
+
+
+class HasCandidate(C.Structure):
+    _fields_ = [("n_encode", C.c_int32), ("n_prefill", C.c_int32), ("n_decode", C.c_int32), ("n_local", C.c_int32),
+                ("rho_e", C.c_double), ("rho_p", C.c_double), ("rho_d", C.c_double), ("score", C.c_double),
+                ("b_max", C.c_int32), ("s_star", C.c_double), ("kept", C.c_int32)]
 
 
 class Router(C.Structure):
@@ -54,6 +60,9 @@ def lib():
                                          C.POINTER(C.c_double), C.POINTER(C.c_double), C.c_double, C.POINTER(SmTable)]
         l.eas_sm_table_lookup.restype = C.c_int32
         l.eas_sm_table_lookup.argtypes = [C.POINTER(SmTable), C.c_int32]
+        l.eas_has_stage1.restype = C.c_int32
+        l.eas_has_stage1.argtypes = [C.POINTER(HasCandidate), C.c_int32, C.c_double, C.c_double, C.c_double, C.c_double,
+                                     C.c_double, C.c_double, C.c_int32]
         _declared = True
     return l
 
@@ -128,3 +137,15 @@ def sm_table_build(sm_counts, batches, latency, exclusive, tol=0.2) -> SmTable:
 
 def sm_table_lookup(t: SmTable, batch: int) -> int:
     return lib().eas_sm_table_lookup(C.byref(t), batch)
+
+
+def has_stage1(cands, rate, c_e, c_p, c_d, alpha, prune=1.2, top_k=3):
+    """cands: [(n_E, n_P, n_D, n_L)] -> (rows (rho_E, rho_P, rho_D, score, B_max, s*), kept indices)."""
+    arr = (HasCandidate * len(cands))()
+    for i, (nE, nP, nD, nL) in enumerate(cands):
+        arr[i].n_encode, arr[i].n_prefill, arr[i].n_decode, arr[i].n_local = nE, nP, nD, nL
+    n = lib().eas_has_stage1(arr, len(cands), rate, c_e, c_p, c_d, alpha, prune, top_k)
+    if n < 0:
+        raise ValueError("bad Stage-1 arguments")
+    rows = [(a.rho_e, a.rho_p, a.rho_d, a.score, a.b_max, a.s_star) for a in arr]
+    return rows, [i for i, a in enumerate(arr) if a.kept]

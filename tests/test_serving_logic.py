@@ -148,3 +148,28 @@ def test_library_router_envelopes_and_table_match_oracle(sv):
     assert [(t.sm_count[i], t.max_batch[i]) for i in range(t.n_levels)] == ref
     for b in range(1, 20):
         assert sv.sm_table_lookup(t, b) == SO.sm_table_lookup(ref, b)
+
+
+def test_has_stage1_oracle_properties_and_library(sv):
+    # 8 GPUs, encode workers on 1 GPU, prefill/decode workers on 2 GPUs each, one local prefill worker per encode GPU
+    cands = [(nE, P // 2, D // 2, nE) for nE in range(1, 7) for P in (0, 2, 4) for D in (2, 4) if nE + P + D == 8]
+    rate, cE, cP, cD, alpha = 2.5, 2.1, 2.0, 3.4, 0.5
+    rows, kept = SO.has_stage1(cands, rate, cE, cP, cD, alpha)
+    for (nE, nP, nD, nL), (rE, rP, rD, score, bmax, s_star) in zip(cands, rows):
+        assert abs(rE - rate / nE / cE) < 1e-15 and abs(rD - rate / nD / cD) < 1e-15            # Eq. 3
+        assert abs(rP - rate / (cP * (nP + nL * alpha))) < 1e-15                                   # prefill with the local term
+        assert score == max(rE, rP, rD) and bmax == math.ceil(rate / nE)                           # Eq. 4, B_max
+        assert abs(s_star - nP * cP / (nP * cP + nL * alpha * cP)) < 1e-15                         # C_remote / (C_remote + C_local)
+    assert 1 <= len(kept) <= 3
+    best = min(r[3] for r in rows if r[3] < 1)
+    assert all(rows[i][3] < 1 and rows[i][3] <= 1.2 * best for i in kept)
+    dropped = [i for i in range(len(cands)) if i not in kept and rows[i][3] < 1 and rows[i][3] <= 1.2 * best]
+    assert all(rows[i][3] >= max(rows[k][3] for k in kept) for i in dropped)                       # only the top K stay
+    # every stage overloaded -> nothing survives
+    assert SO.has_stage1(cands, 500.0, cE, cP, cD, alpha)[1] == []
+    lrows, lkept = sv.has_stage1(cands, rate, cE, cP, cD, alpha)
+    assert lkept == kept
+    assert np.allclose(np.asarray(lrows, dtype=float), np.asarray(rows, dtype=float), rtol=0, atol=1e-14)
+    assert sv.has_stage1(cands, 500.0, cE, cP, cD, alpha)[1] == []
+    with pytest.raises(ValueError):
+        sv.has_stage1([(0, 1, 1, 0)], rate, cE, cP, cD, alpha)
