@@ -48,10 +48,17 @@ struct AttnTcSmem {
   static constexpr int kHiBytes = kTcTile * HI * 2;        // 128 rows x 16 bf16
   static constexpr int kTileBytes = kLoBytes + kHiBytes;   // one Q, K or V tile
   static constexpr bool kStagedOut = PT && HD == 64;       // output rows leave through shared memory and TMA stores
-  static constexpr int kStages = PT ? (HD == 64 ? 4 : 3) : (HD == 64 ? 3 : 2);
+  // With P in tensor memory and head_dim 80, V is loaded 128 columns wide (two 64-column boxes; the extra 48 columns
+  // belong to the next head, or are zero past the last one) so that P V is ONE N = 128 UMMA per 16 keys instead of an
+  // N = 64 plus an N = 16 one: the issuer is the bottleneck there and every UMMA costs about the same.  The surplus
+  // output columns 80..127 of O are never read.
+  static constexpr bool kWideV = PT && HD != 64;
+  static constexpr int kVBytes = kWideV ? 2 * kLoBytes : kTileBytes;
+  static constexpr int kStageBytes = kTileBytes + kVBytes;  // K then V
+  static constexpr int kStages = PT ? (HD == 64 ? 4 : 2) : (HD == 64 ? 3 : 2);
   static constexpr int kQOff = 0;                          // [2 buffers][2 tiles]
   static constexpr int kKvOff = kQOff + 4 * kTileBytes;    // [stages][K, V]
-  static constexpr int kPOff = kKvOff + kStages * 2 * kTileBytes;   // [2 tiles][2 k-blocks of 16 KB] (shared-memory P only)
+  static constexpr int kPOff = kKvOff + kStages * kStageBytes;   // [2 tiles][2 k-blocks of 16 KB] (shared-memory P only)
   static constexpr int kOutOff = kPOff + (PT ? 0 : 2 * 32768);      // [8 softmax warps][32 rows x 128 bytes]
   static constexpr int kBarOff = kOutOff + (kStagedOut ? 8 * 4096 : 0);
   static constexpr int kBytes = kBarOff + 512 + 1024;      // barriers + alignment slack
@@ -223,8 +230,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_tc_kernel(const __grid_con
   pdl_wait();
 
   auto q_tile = [&](int buf, int t) { return smem + L::kQOff + (buf * 2 + t) * L::kTileBytes; };
-  auto k_tile = [&](int s) { return smem + L::kKvOff + (s * 2) * L::kTileBytes; };
-  auto v_tile = [&](int s) { return smem + L::kKvOff + (s * 2 + 1) * L::kTileBytes; };
+  auto k_tile = [&](int s) { return smem + L::kKvOff + s * L::kStageBytes; };
+  auto v_tile = [&](int s) { return smem + L::kKvOff + s * L::kStageBytes + L::kTileBytes; };
   auto p_tile = [&](int w) { return smem + L::kPOff + w * 32768; };
 
   if (warp == 0) {
@@ -252,9 +259,10 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_tc_kernel(const __grid_con
           mbar_expect_tx(&k_full[s], L::kTileBytes);
           tma_load_2d(k_tile(s), &p.map_lo, &k_full[s], p.d_model + xq, y);
           if (HI) tma_load_2d(k_tile(s) + L::kLoBytes, &p.map_hi, &k_full[s], p.d_model + xq + 64, y);
-          mbar_expect_tx(&v_full[s], L::kTileBytes);
+          mbar_expect_tx(&v_full[s], L::kVBytes);
           tma_load_2d(v_tile(s), &p.map_lo, &v_full[s], 2 * p.d_model + xq, y);
-          if (HI) tma_load_2d(v_tile(s) + L::kLoBytes, &p.map_hi, &v_full[s], 2 * p.d_model + xq + 64, y);
+          if (L::kWideV) tma_load_2d(v_tile(s) + L::kLoBytes, &p.map_lo, &v_full[s], 2 * p.d_model + xq + 64, y);
+          else if (HI) tma_load_2d(v_tile(s) + L::kLoBytes, &p.map_hi, &v_full[s], 2 * p.d_model + xq + 64, y);
         }
       }
       if (!ok) {
@@ -269,6 +277,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_tc_kernel(const __grid_con
       constexpr uint32_t idesc_s = make_idesc_bf16(128, 128, 0, 0);     // S = Q K^T, both K-major
       constexpr uint32_t idesc_o_lo = make_idesc_bf16(128, 64, 0, 1);   // O[:, 0:64] += P V, V is MN-major
       constexpr uint32_t idesc_o_hi = make_idesc_bf16(128, 16, 0, 1);   // O[:, 64:80]
+      constexpr uint32_t idesc_o_wide = make_idesc_bf16(128, 128, 0, 1); // O[:, 0:128] from the 128-column V tile
       uint32_t kv_it = 0, u_cnt = 0;
       uint32_t n_tiles[2] = {0, 0};            // S tiles issued per warpgroup (phase counters)
       uint32_t n_pv[2] = {0, 0};
@@ -297,7 +306,12 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_tc_kernel(const __grid_con
         for (int ks = 0; ks < 8; ++ks) {       // 16 keys per step
           const uint64_t bd = make_smem_desc(va + ks * 2048, 1024, 1024, kSwizzle128B);
           const uint32_t acc = (accumulate || ks != 0) ? 1u : 0u;
-          if (PT) {
+          if (L::kWideV) {
+            // two 64-column swizzle atoms 16 KB apart (leading byte offset), 8-key groups 1 KB apart
+            const uint32_t pt = tmem_base + L::kPCol0 + w * L::kPStride + ks * 8;
+            const uint64_t bw = make_smem_desc(va + ks * 2048, L::kLoBytes, 1024, kSwizzle128B);
+            umma_bf16_ts(d, pt, bw, idesc_o_wide, acc);
+          } else if (PT) {
             const uint32_t pt = tmem_base + L::kPCol0 + w * L::kPStride + ks * 8;   // 16 bf16 = 8 columns
             umma_bf16_ts(d, pt, bd, idesc_o_lo, acc);
             if (HI) {
