@@ -154,7 +154,9 @@ def run_reference(args):
     line = {"impl": "reference", "metric": "encoder_tokens_per_sec", "value": val, "unit": "tokens/s", "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": f"{args.config} micro-batch {args.micro_batch} (sample: 1 item per step)"},
+            "config": {"workload": f"{args.config} micro-batch {args.micro_batch}", "items_per_step": len(shapes),
+                       "tokens_per_step": sum(S.tokens_per_item(cfg, s) for s in shapes), "sm_budget": "host cores",
+                       "sampled": "each step encodes 1 item of the micro-batch (bounded sample)"},
             "cpu_baseline": {"value": val, "unit": "tokens/s", "cores": torch.get_num_threads(), "kind": "oracle",
                              "sample": f"1 item ({f['tokens']} tokens) of the {args.config} micro-batch per step"},
             "e2e": {"value": val, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
