@@ -247,24 +247,29 @@ static eas_status finish_linear(Linear& L) {
 }
 
 typedef void (*GemmKernel)(GemmParams);
+// ctas: 1 = one CTA per 128x256 tile; 2 = CTA pair per 256x256 tile; 3 = CTA pair per 256x512 tile ("wide")
 static GemmKernel gemm_kernel_for(int act, int out_fp32, int ctas) {
-  if (ctas == 2) {
-    if (act == ACT_NONE && !out_fp32) return gemm_kernel<ACT_NONE, OUT_BF16, 2>;
-    if (act == ACT_GELU && !out_fp32) return gemm_kernel<ACT_GELU, OUT_BF16, 2>;
-    if (act == ACT_SWIGLU && !out_fp32) return gemm_kernel<ACT_SWIGLU, OUT_BF16, 2>;
-    if (act == ACT_NONE && out_fp32) return gemm_kernel<ACT_NONE, OUT_F32, 2>;
-    if (act == ACT_GELU && out_fp32) return gemm_kernel<ACT_GELU, OUT_F32, 2>;
+  if (ctas == 3) {
+    if (act == ACT_NONE && !out_fp32) return gemm_kernel<ACT_NONE, OUT_BF16, 2, 2>;
+    if (act == ACT_GELU && !out_fp32) return gemm_kernel<ACT_GELU, OUT_BF16, 2, 2>;
+    if (act == ACT_NONE && out_fp32) return gemm_kernel<ACT_NONE, OUT_F32, 2, 2>;
+  } else if (ctas == 2) {
+    if (act == ACT_NONE && !out_fp32) return gemm_kernel<ACT_NONE, OUT_BF16, 2, 1>;
+    if (act == ACT_GELU && !out_fp32) return gemm_kernel<ACT_GELU, OUT_BF16, 2, 1>;
+    if (act == ACT_SWIGLU && !out_fp32) return gemm_kernel<ACT_SWIGLU, OUT_BF16, 2, 1>;
+    if (act == ACT_NONE && out_fp32) return gemm_kernel<ACT_NONE, OUT_F32, 2, 1>;
+    if (act == ACT_GELU && out_fp32) return gemm_kernel<ACT_GELU, OUT_F32, 2, 1>;
   } else {
-    if (act == ACT_NONE && !out_fp32) return gemm_kernel<ACT_NONE, OUT_BF16, 1>;
-    if (act == ACT_GELU && !out_fp32) return gemm_kernel<ACT_GELU, OUT_BF16, 1>;
-    if (act == ACT_SWIGLU && !out_fp32) return gemm_kernel<ACT_SWIGLU, OUT_BF16, 1>;
-    if (act == ACT_NONE && out_fp32) return gemm_kernel<ACT_NONE, OUT_F32, 1>;
-    if (act == ACT_GELU && out_fp32) return gemm_kernel<ACT_GELU, OUT_F32, 1>;
+    if (act == ACT_NONE && !out_fp32) return gemm_kernel<ACT_NONE, OUT_BF16, 1, 1>;
+    if (act == ACT_GELU && !out_fp32) return gemm_kernel<ACT_GELU, OUT_BF16, 1, 1>;
+    if (act == ACT_SWIGLU && !out_fp32) return gemm_kernel<ACT_SWIGLU, OUT_BF16, 1, 1>;
+    if (act == ACT_NONE && out_fp32) return gemm_kernel<ACT_NONE, OUT_F32, 1, 1>;
+    if (act == ACT_GELU && out_fp32) return gemm_kernel<ACT_GELU, OUT_F32, 1, 1>;
   }
   return nullptr;
 }
 static eas_status set_kernel_attributes() {
-  for (int ctas = 1; ctas <= 2; ++ctas)
+  for (int ctas = 1; ctas <= 3; ++ctas)
     for (int act = 0; act < 3; ++act)
       for (int f32 = 0; f32 < 2; ++f32) {
         GemmKernel k = gemm_kernel_for(act, f32, ctas);
@@ -539,6 +544,12 @@ static eas_status launch_gemm(const GemmCall& g, int budget, cudaStream_t stream
   if (L.N % 32 != 0 || g.a_run % kBK != 0) return fail(EAS_ERR_UNSUPPORTED, "GEMM needs N %% 32 == 0 and K %% 64 == 0 (N=%d, K=%lld)", L.N, static_cast<long long>(g.a_run));
   // CTA pairs (two SMs on one 256x256 tile, each loading half of the weight tile) whenever two SMs are available
   const int ctas = budget >= 2 ? 2 : 1;
+  const bool tma_out = g.row_map == nullptr && g.pos == nullptr && (g.resid == nullptr || g.resid == g.out);
+  // wide 256x512 tiles for long reductions whose output splits evenly into 512-column blocks
+  const int64_t k_total = g.a_run * g.taps;
+  const bool wide = ctas == 2 && tma_out && g.act != ACT_SWIGLU && k_total >= 2048 && L.N % 512 == 0 &&
+                    gemm_kernel_for(g.act, g.out_fp32, 3) != nullptr;
+  const int tile_n = wide ? 2 * kBN : kBN;
   GemmParams p{};
   EAS_TRY(make_a_tmap(&p.tma_a, g.A, g.a_run, g.a_row_elems, g.conv_stride, g.a_rows));
   p.tma_b = ctas == 2 ? L.tmap_half : L.tmap;
@@ -547,20 +558,20 @@ static eas_status launch_gemm(const GemmCall& g, int budget, cudaStream_t stream
   p.k_blocks = p.kb_per_tap * g.taps;
   p.conv_stride = g.conv_stride;
   p.m_blocks = (g.M + kBM * ctas - 1) / (kBM * ctas);
-  p.n_blocks = (L.N + kBN - 1) / kBN;
+  p.n_blocks = (L.N + tile_n - 1) / tile_n;
   p.bias = L.b;
   p.out = g.out; p.ldo = g.ldo; p.resid = g.resid;
   p.row_map = g.row_map; p.pos_idx = g.pos_idx; p.pos = g.pos;
   p.rope_cs = g.rope_cs; p.rope_pairs = g.rope_pairs; p.rope_ncols = g.rope_ncols; p.head_dim = g.head_dim > 0 ? g.head_dim : 64;
   p.status = status;
   // TMA-store epilogue whenever output rows are the A rows and any residual is accumulated in place
-  p.use_tma_out = (g.row_map == nullptr && g.pos == nullptr && (g.resid == nullptr || g.resid == g.out)) ? 1 : 0;
+  p.use_tma_out = tma_out ? 1 : 0;
   if (p.use_tma_out) {
     const int64_t out_cols = g.act == ACT_SWIGLU ? L.N / 2 : L.N;
     EAS_TRY(make_out_tmap(&p.tma_out, g.out, g.out_fp32 != 0, out_cols, g.ldo, g.M));
   }
   const int tiles = p.m_blocks * p.n_blocks;
-  GemmKernel kern = gemm_kernel_for(g.act, g.out_fp32, ctas);
+  GemmKernel kern = gemm_kernel_for(g.act, g.out_fp32, wide ? 3 : ctas);
   if (kern == nullptr) return fail(EAS_ERR_UNSUPPORTED, "no GEMM epilogue for act=%d out_fp32=%d", g.act, g.out_fp32);
   return launch_kernel(kern, std::min(budget / ctas, tiles) * ctas, kGemmThreads, kGemmSmemBytes, stream, p, ctas);
 }

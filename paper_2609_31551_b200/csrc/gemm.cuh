@@ -20,10 +20,14 @@ constexpr int kGemmThreads = 64 + 32 * kEpiWarps;
 constexpr int kABytes = kBM * kBK * 2;            // 16 KB: 128 rows of A
 // one CTA per tile: a stage holds A (16 KB) + the whole 256-row weight tile (32 KB), 4 stages;
 // CTA pair per 256x256 tile: a stage holds A (16 KB) + this CTA's 128 weight rows (16 KB), 6 stages
-template <int CTAS> struct GemmCfg {
-  static constexpr int kBBytes = (kBN / CTAS) * kBK * 2;
+// NW = 2 ("wide", CTA pairs only): the pair owns a 256x512 tile, i.e. two 256-column accumulators fed by the same
+// A tile.  That cuts the operand bytes per FLOP by a quarter (the L2 -> SM path is what bounds the main loop) at the
+// price of a single accumulator set: the epilogue no longer overlaps the next main loop, so it pays for large K only.
+template <int CTAS, int NW> struct GemmCfg {
+  static constexpr int kBBytes = (kBN / CTAS) * kBK * 2 * NW;
   static constexpr int kStageBytes = kABytes + kBBytes;
-  static constexpr int kStages = CTAS == 2 ? 6 : 4;
+  static constexpr int kStages = CTAS == 2 ? (NW == 2 ? 4 : 6) : 4;
+  static constexpr int kAccBuffers = NW == 2 ? 1 : 2;
 };
 constexpr int kMaxStages = 6;
 constexpr int kStagingOff = 4 * 49152;                         // == 6 * 32768; 8 epilogue warps x 4 KB output staging (TMA store source)
@@ -70,10 +74,13 @@ __device__ __forceinline__ void tile_coords(int tile, int m_blocks, int n_blocks
   mb = panel * kPanelM + (within - nb * rows_here);
 }
 
-template <int ACT, int OUT, int CTAS>
+template <int ACT, int OUT, int CTAS, int NW>
 __global__ void __launch_bounds__(kGemmThreads, 1) gemm_kernel(const __grid_constant__ GemmParams p) {
-  constexpr int kStages = GemmCfg<CTAS>::kStages;
-  constexpr int kStageBytes = GemmCfg<CTAS>::kStageBytes;
+  static_assert(NW == 1 || (CTAS == 2 && ACT != ACT_SWIGLU), "wide tiles: CTA pairs, no gated epilogue");
+  constexpr int kStages = GemmCfg<CTAS, NW>::kStages;
+  constexpr int kStageBytes = GemmCfg<CTAS, NW>::kStageBytes;
+  constexpr int kAccBuffers = GemmCfg<CTAS, NW>::kAccBuffers;
+  constexpr int kTileN = kBN * NW;                 // output columns of a tile
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   // 1024-byte alignment: the 128-byte swizzle pattern repeats every 8 rows of 128 bytes
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -135,7 +142,10 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_kernel(const __grid_cons
             // both CTAs' loads complete on the leader's barrier; the leader announces the bytes of both
             if (cta_rank == 0) mbar_expect_tx(&full_bar[s], 2 * kStageBytes);
             tma_load_3d_pair(sa, &p.tma_a, &full_bar[s], kx, tap % p.conv_stride, mb * kBM + tap / p.conv_stride);
-            tma_load_2d_pair(sb, &p.tma_b, &full_bar[s], kb * kBK, nb * kBN + cta_rank * (kBN / 2));
+#pragma unroll
+            for (int h = 0; h < NW; ++h)
+              tma_load_2d_pair(sb + h * (kBN / 2) * kBK * 2, &p.tma_b, &full_bar[s], kb * kBK,
+                               nb * kTileN + h * kBN + cta_rank * (kBN / 2));
           } else {
             mbar_expect_tx(&full_bar[s], kStageBytes);
             tma_load_3d(sa, &p.tma_a, &full_bar[s], kx, tap % p.conv_stride, mb * kBM + tap / p.conv_stride);
@@ -158,8 +168,8 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_kernel(const __grid_cons
       uint32_t it = 0, tcount = 0;
       bool ok = true;
       for (int tile = first_tile; tile < num_tiles && ok; tile += tile_step, ++tcount) {
-        const uint32_t acc = tcount & 1u;
-        const uint32_t acc_ph = (tcount >> 1) & 1u;
+        const uint32_t acc = tcount % kAccBuffers;
+        const uint32_t acc_ph = (tcount / kAccBuffers) & 1u;
         if (!mbar_wait(&acc_empty[acc], acc_ph ^ 1u, abort_flag)) { ok = false; break; }
         tc_fence_after_sync();
         const uint32_t tmem_d = tmem_base + acc * kBN;
@@ -175,8 +185,14 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_kernel(const __grid_cons
 #pragma unroll
           for (int k = 0; k < kBK / 16; ++k) {
             // advancing 16 bf16 = 32 bytes along K inside the swizzle atom: +2 in the (>>4) address field
-            if (CTAS == 2) umma_bf16_ss_pair(tmem_d, adesc + 2 * k, bdesc + 2 * k, idesc, (kb | k) != 0);
-            else umma_bf16_ss(tmem_d, adesc + 2 * k, bdesc + 2 * k, idesc, (kb | k) != 0);
+            if (CTAS == 2) {
+#pragma unroll
+              for (int h = 0; h < NW; ++h)   // second accumulator: the next 128 weight rows of each CTA, 16 KB further
+                umma_bf16_ss_pair(tmem_d + h * kBN, adesc + 2 * k, bdesc + 2 * k + h * ((kBN / 2) * kBK * 2 / 16), idesc,
+                                  (kb | k) != 0);
+            } else {
+              umma_bf16_ss(tmem_d, adesc + 2 * k, bdesc + 2 * k, idesc, (kb | k) != 0);
+            }
           }
           // frees the stage (in both CTAs of a pair) once these UMMAs have read it
           if (CTAS == 2) umma_commit_pair_multicast(&empty_bar[s], 3); else umma_commit(&empty_bar[s]);
@@ -204,15 +220,18 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_kernel(const __grid_cons
       int mg, nb;
       tile_coords(tile, p.m_blocks, p.n_blocks, mg, nb);
       const int mb = mg * CTAS + cta_rank;
-      const uint32_t acc = tcount & 1u;
-      const uint32_t acc_ph = (tcount >> 1) & 1u;
+      const uint32_t acc = tcount % kAccBuffers;
+      const uint32_t acc_ph = (tcount / kAccBuffers) & 1u;
       if (p.use_tma_out) {
         // ---- staged path: bias from shared memory, 32-row sub-tiles written to a swizzled staging buffer
         //      and stored (or reduce-added, for the fp32 residual stream) by TMA; rows >= M are clipped by TMA
-        float* sbias = reinterpret_cast<float*>(smem + kBiasOff) + acc * 256;
+        float* sbias = reinterpret_cast<float*>(smem + kBiasOff) + acc * 256;   // wide tiles use both halves as one
         {
-          const int col = nb * kBN + ew * 32 + lane;
-          sbias[ew * 32 + lane] = col < p.N ? __bfloat162float(p.bias[col]) : 0.f;
+#pragma unroll
+          for (int h = 0; h < NW; ++h) {
+            const int col = nb * kTileN + h * 256 + ew * 32 + lane;
+            sbias[h * 256 + ew * 32 + lane] = col < p.N ? __bfloat162float(p.bias[col]) : 0.f;
+          }
           __syncwarp();
           if (lane == 0) mbar_arrive(&bias_bar[acc]);
         }
@@ -223,12 +242,12 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_kernel(const __grid_cons
         uint8_t* srow = stage + lane * 128;
         const int sw = lane & 7;
         const int arow = mb * kBM + quarter * 32 + lane;
-        const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + acc * kBN + half * 128;
+        const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + acc * kBN + half * (128 * NW);
         const int ycoord = mb * kBM + quarter * 32;
 
         auto finish_chunk = [&](float (&v)[32], int c) {   // bias, rotary, activation on 32 accumulator columns
-          const int col0 = nb * kBN + half * 128 + c * 32;
-          const float4* b4 = reinterpret_cast<const float4*>(sbias + half * 128 + c * 32);
+          const int col0 = nb * kTileN + half * (128 * NW) + c * 32;
+          const float4* b4 = reinterpret_cast<const float4*>(sbias + half * (128 * NW) + c * 32);
 #pragma unroll
           for (int q = 0; q < 8; ++q) {
             const float4 b = b4[q];
@@ -271,7 +290,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_kernel(const __grid_cons
         };
 
 #pragma unroll 1
-        for (int pr = 0; pr < 2; ++pr) {            // two chunks (64 accumulator columns) per round
+        for (int pr = 0; pr < 2 * NW; ++pr) {       // two chunks (64 accumulator columns) per round
           uint32_t r0[32], r1[32];
           __syncwarp();
           tmem_ld_32x32(taddr + pr * 64, r0);
@@ -282,7 +301,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_kernel(const __grid_cons
           for (int i = 0; i < 32; ++i) { v0[i] = __uint_as_float(r0[i]); v1[i] = __uint_as_float(r1[i]); }
           finish_chunk(v0, pr * 2);
           finish_chunk(v1, pr * 2 + 1);
-          const int col0 = nb * kBN + half * 128 + pr * 64;
+          const int col0 = nb * kTileN + half * (128 * NW) + pr * 64;
           if (OUT == OUT_F32) {
             // 32 fp32 columns = one 128-byte staging row; two sub-tiles per round
 #pragma unroll

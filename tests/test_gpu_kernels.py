@@ -19,7 +19,8 @@ def _dev(a):
 
 
 @pytest.mark.parametrize("M,N,K", [(784, 256, 768), (300, 512, 128), (129, 256, 64), (1, 32, 64), (257, 96, 640),
-                                   (1000, 1024, 1024), (128, 3072, 256), (77, 288, 192)])
+                                   (1000, 1024, 1024), (128, 3072, 256), (77, 288, 192),
+                                   (300, 1024, 2048), (1000, 512, 4096)])   # the last two take the wide 256x512 tiles
 @pytest.mark.parametrize("act,out_fp32", [(0, False), (1, False), (2, False), (0, True)])
 def test_gemm_epilogues(M, N, K, act, out_fp32):
     import paper_2609_31551_b200 as P
@@ -45,7 +46,7 @@ def test_gemm_epilogues(M, N, K, act, out_fp32):
     assert not bad.any(), f"{int(bad.sum())} of {bad.numel()} wrong, max err {(got - y).abs().max():.4e}, first bad {bad.nonzero()[:5].tolist()}"
 
 
-@pytest.mark.parametrize("M,N,K", [(300, 512, 128), (1000, 1024, 1024), (77, 288, 192)])
+@pytest.mark.parametrize("M,N,K", [(300, 512, 128), (1000, 1024, 1024), (77, 288, 192), (513, 1024, 2048), (700, 1536, 4096)])
 def test_gemm_residual_accumulated_in_place(M, N, K):
     """fp32 residual stream updated in place (x += A W^T + b): the path the encoder's proj / fc2 GEMMs take."""
     import paper_2609_31551_b200 as P
