@@ -62,10 +62,11 @@ def test_gemm_residual_accumulated_in_place(M, N, K):
     assert err.max() <= 1e-5 * float(y.abs().max()) + 2e-3 * max(1.0, float(K) ** 0.5 * 0.05), err.max()
 
 
-def test_gemm_is_independent_of_sm_budget():
+@pytest.mark.parametrize("N,K", [(768, 512), (1024, 2048)])      # narrow 256x256 tiles; wide 256x512 tiles
+def test_gemm_is_independent_of_sm_budget(N, K):
     import paper_2609_31551_b200 as P
     rng = np.random.Generator(np.random.PCG64(5))
-    A, W, b = _dev(_bf16_exact(rng, (1500, 512))), _dev(_bf16_exact(rng, (768, 512), 0.05)), _dev(_bf16_exact(rng, (768,)))
+    A, W, b = _dev(_bf16_exact(rng, (1500, K))), _dev(_bf16_exact(rng, (N, K), 0.05)), _dev(_bf16_exact(rng, (N,)))
     ref, _ = P.kernel_gemm(A, W, b, act=1)
     for budget in (1, 7, 37, 74, 111):
         out, _ = P.kernel_gemm(A, W, b, act=1, sm_budget=budget)
