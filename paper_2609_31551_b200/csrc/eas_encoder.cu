@@ -547,8 +547,18 @@ static eas_status launch_gemm(const GemmCall& g, int budget, cudaStream_t stream
   const bool tma_out = g.row_map == nullptr && g.pos == nullptr && (g.resid == nullptr || g.resid == g.out);
   // wide 256x512 tiles for long reductions whose output splits evenly into 512-column blocks
   const int64_t k_total = g.a_run * g.taps;
-  const bool wide = ctas == 2 && tma_out && g.act != ACT_SWIGLU && k_total >= 2048 && L.N % 512 == 0 &&
-                    gemm_kernel_for(g.act, g.out_fp32, 3) != nullptr;
+  bool wide = ctas == 2 && tma_out && g.act != ACT_SWIGLU && k_total >= 2048 && L.N % 512 == 0 &&
+              gemm_kernel_for(g.act, g.out_fp32, 3) != nullptr;
+  if (wide) {
+    // only when the half as many, twice as large tiles still fill the CTA pairs about as evenly (a wide tile is worth
+    // roughly 15 % per unit of work); the two tilings give bit-identical results, so this is a pure speed choice
+    const long long pairs = budget / 2;
+    const long long mg = (g.M + 2 * kBM - 1) / (2 * kBM);
+    const long long t_n = mg * ((L.N + kBN - 1) / kBN), t_w = mg * (L.N / (2 * kBN));
+    const double eff_n = static_cast<double>(t_n) / static_cast<double>(((t_n + pairs - 1) / pairs) * pairs);
+    const double eff_w = static_cast<double>(t_w) / static_cast<double>(((t_w + pairs - 1) / pairs) * pairs);
+    wide = t_w >= pairs && eff_w * 1.15 >= eff_n;
+  }
   const int tile_n = wide ? 2 * kBN : kBN;
   GemmParams p{};
   EAS_TRY(make_a_tmap(&p.tma_a, g.A, g.a_run, g.a_row_elems, g.conv_stride, g.a_rows));
