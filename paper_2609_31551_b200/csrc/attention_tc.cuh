@@ -480,6 +480,9 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_tc_kernel(const __grid_con
       float m_used = -INFINITY, l = 0.f;
       for (int j = 0; j < u.n_kv; ++j, ++n) {
         ATTN_STAMP(0);
+        // The previous unit's output goes out here: its last P V was issued before this unit's first scores,
+        // so it is complete while those are still being computed, and the write hides behind that wait.
+        if (j == 0 && pend && !flush_output()) { ok = false; break; }
         if (!mbar_wait(&s_full[w], n & 1u, abort_flag)) { ok = false; break; }
         tc_fence_after_sync();
         ATTN_STAMP(1);
@@ -553,7 +556,6 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_tc_kernel(const __grid_con
         // S has been read: the issuer may overwrite it with the next tile's scores once p_ready fires.
         // The previous P V must be complete before P is overwritten or O is touched.
         ATTN_STAMP(4);
-        if (j == 0 && pend && !flush_output()) { ok = false; break; }
         if (n > 0 && !mbar_wait(&pv_done[w], (n - 1) & 1u, abort_flag)) { ok = false; break; }
         ATTN_STAMP(5);
         tc_fence_after_sync();
