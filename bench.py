@@ -185,6 +185,10 @@ def run_cuda(args):
     f = flops_of(cfg, shapes)
     T = f["tokens"]
     budget = args.sm_budget
+    if args.graph:
+        # the launch-overhead path: captured forward passes need a stream of their own
+        torch.cuda.set_stream(torch.cuda.Stream())
+        enc.set_graph_mode(True)
     stream = torch.cuda.current_stream()
     out = torch.empty((f["out_rows"], cfg["d_out"]), dtype=torch.bfloat16, device="cuda")
 
@@ -299,7 +303,8 @@ def run_cuda(args):
             "config": {"workload": f"{args.config} micro-batch {args.micro_batch}", "items_per_step": len(shapes),
                        "tokens_per_step": T, "sm_budget": budget if budget else "all",
                        "l2": "working set (weights + activations) larger than L2; no flush",
-                       "parallelism": "replicas" if world > 1 else "single"},
+                       "parallelism": "replicas" if world > 1 else "single",
+                       "launch": "cuda graph replay" if args.graph else "one launch per kernel"},
             "items_per_sec": total_items * args.steps / (ms * 1e-3),
             "tflops": total_flops / (step_ms * 1e-3) / 1e12,
             "frac_of_bf16_peak": {"burst_measured": f["total"] / (step_ms * 1e-3) / 1e12 / peaks["burst"],
@@ -354,6 +359,8 @@ def main():
     ap.add_argument("--micro-batch", type=int, default=32)
     ap.add_argument("--sm-budget", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--graph", action="store_true",
+                    help="replay captured forward passes (CUDA graphs): the launch-overhead path for small micro-batches")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

@@ -168,6 +168,21 @@ int32_t eas_encoder_last_launch_count(const eas_encoder* enc);
  * testing. */
 eas_status eas_encoder_set_attention_impl(eas_encoder* enc, int32_t impl);
 
+/* Launch-overhead path for small micro-batches (Section 3.2: a forward pass at small batch size is dominated by
+ * kernel-launch and scheduling overhead).  mode 1: eas_encode_microbatch / _static capture the launches of a
+ * micro-batch into a CUDA graph the first time they see it and replay the graph afterwards (one driver call per
+ * forward pass instead of one per kernel).  A micro-batch is "the same" when n_items, item_shape, item_offset,
+ * cu_seqlens_host, sm_budget, the attention variant and every pointer (data, workspace, cu_seqlens_dev,
+ * out_embeddings) are equal; the VALUES behind the pointers may change freely.  The kernels and their arguments are
+ * those of the ordinary path, so results are bit-identical.  Up to 16 captures are kept per encoder (least recently
+ * used goes first); mode 0 (default) drops them.  Capture needs a real stream: with the NULL / legacy / per-thread
+ * default stream, while per-kernel timing is on, or while the caller is itself capturing `stream`, calls run
+ * uncaptured.  The cached graphs refer to the caller's buffers: do not free those while the mode is on. */
+eas_status eas_encoder_set_graph_mode(eas_encoder* enc, int32_t mode);
+
+/* Counters of the graph path: replays, captures, and captures currently held (any pointer may be NULL). */
+eas_status eas_encoder_graph_stats(const eas_encoder* enc, int64_t* hits, int64_t* captures, int32_t* cached);
+
 /* Per-kernel timing for profiling (off by default; adds one event record per launch).  Kernel classes: */
 enum { EAS_KC_PREP = 0, EAS_KC_EMBED_GATHER = 1, EAS_KC_GEMM_EMBED = 2, EAS_KC_NORM = 3, EAS_KC_GEMM_QKV = 4,
        EAS_KC_ATTENTION = 5, EAS_KC_GEMM_PROJ = 6, EAS_KC_GEMM_FC1 = 7, EAS_KC_GEMM_FC2 = 8, EAS_KC_GEMM_HEAD = 9,

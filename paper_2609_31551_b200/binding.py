@@ -16,7 +16,7 @@ STATUS_NAMES = {0: "EAS_OK", 1: "EAS_ERR_INVALID_ARG", 2: "EAS_ERR_UNSUPPORTED",
 EXPORTED_SYMBOLS = [
     "eas_encoder_create", "eas_encoder_weight_arena_bytes", "eas_encoder_workspace_bytes", "eas_encoder_out_rows",
     "eas_encode_microbatch", "eas_encode_microbatch_static", "eas_encoder_status", "eas_encoder_last_launch_count", "eas_encoder_set_attention_impl",
-    "eas_encoder_enable_timing", "eas_encoder_timing_read", "eas_last_error", "eas_encoder_destroy", "eas_kernel_gemm", "eas_kernel_norm", "eas_kernel_attention",
+    "eas_encoder_set_graph_mode", "eas_encoder_graph_stats", "eas_encoder_enable_timing", "eas_encoder_timing_read", "eas_last_error", "eas_encoder_destroy", "eas_kernel_gemm", "eas_kernel_norm", "eas_kernel_attention",
 ]
 
 
@@ -77,6 +77,10 @@ def load_library():
     lib.eas_encoder_last_launch_count.argtypes = [C.c_void_p]
     lib.eas_encoder_set_attention_impl.restype = C.c_int
     lib.eas_encoder_set_attention_impl.argtypes = [C.c_void_p, C.c_int32]
+    lib.eas_encoder_set_graph_mode.restype = C.c_int
+    lib.eas_encoder_set_graph_mode.argtypes = [C.c_void_p, C.c_int32]
+    lib.eas_encoder_graph_stats.restype = C.c_int
+    lib.eas_encoder_graph_stats.argtypes = [C.c_void_p, C.POINTER(C.c_int64), C.POINTER(C.c_int64), C.POINTER(C.c_int32)]
     lib.eas_encoder_enable_timing.restype = C.c_int
     lib.eas_encoder_enable_timing.argtypes = [C.c_void_p, C.c_int32]
     lib.eas_encoder_timing_read.restype = C.c_int32
@@ -231,6 +235,16 @@ class Encoder:
         _check(self.lib.eas_encode_microbatch_static(self.handle, C.byref(pin), cu_seqlens_dev.data_ptr(), sm_budget,
                                                      _stream_ptr(stream), out.data_ptr()))
         return out
+
+    def set_graph_mode(self, on: bool):
+        """eas_encoder_set_graph_mode: replay captured forward passes for repeated micro-batch shapes.  Needs a
+        non-default stream, and the same data / cu_seqlens_dev / out / workspace tensors from call to call."""
+        _check(self.lib.eas_encoder_set_graph_mode(self.handle, int(on)))
+
+    def graph_stats(self) -> dict:
+        h, c, n = C.c_int64(0), C.c_int64(0), C.c_int32(0)
+        _check(self.lib.eas_encoder_graph_stats(self.handle, C.byref(h), C.byref(c), C.byref(n)))
+        return {"hits": h.value, "captures": c.value, "cached": n.value}
 
     def status(self, stream=None):
         """eas_encoder_status: synchronises the stream and raises on a device-side error."""

@@ -115,6 +115,16 @@ struct Layer {
   Linear qkv, proj, fc1, fc2;
 };
 
+// One captured forward pass: every launch of a micro-batch with exactly these shapes, pointers and SM budget.
+struct GraphEntry {
+  std::vector<int64_t> key;
+  cudaGraphExec_t exec = nullptr;
+  int launches = 0;
+  uint32_t* status = nullptr;
+  uint64_t last_use = 0;
+};
+constexpr size_t kMaxGraphs = 16;
+
 struct eas_encoder {
   eas_arch_config cfg;
   int sm_count = 0;
@@ -130,8 +140,14 @@ struct eas_encoder {
   bool timing = false;
   std::vector<cudaEvent_t> tev;
   std::vector<int> tcls;
+  // optional replay of captured forward passes (small micro-batches are bound by launch overhead)
+  int graph_mode = 0;
+  std::vector<GraphEntry> graphs;
+  uint64_t graph_clock = 0;
+  int64_t graph_hits = 0, graph_captures = 0;
   ~eas_encoder() {
     for (cudaEvent_t ev : tev) cudaEventDestroy(ev);
+    for (GraphEntry& g : graphs) if (g.exec) cudaGraphExecDestroy(g.exec);
   }
 };
 
@@ -935,10 +951,104 @@ static eas_status encode_impl(eas_encoder* e, const eas_packed_inputs* in, void*
   return EAS_OK;
 }
 
+// The forward pass through the graph cache.  A micro-batch is identified by everything the launches depend on:
+// item shapes and offsets, cu_seqlens, the SM budget, the attention variant and every pointer.  A hit replays the
+// captured launches (one driver call instead of one per kernel); a miss captures them from the ordinary code path,
+// so the kernels and their arguments are the same either way.
+static eas_status encode_cached(eas_encoder* e, const eas_packed_inputs* in, void* workspace, size_t workspace_bytes,
+                                const int32_t* cu_dev, int32_t sm_budget, void* stream_v, void* out_embeddings) {
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+  const bool usable = e != nullptr && e->graph_mode != 0 && !e->timing && in != nullptr && in->item_shape != nullptr &&
+                      in->item_offset != nullptr && in->cu_seqlens_host != nullptr && in->n_items >= 1 &&
+                      in->n_items <= EAS_MAX_ITEMS && stream != nullptr && stream != cudaStreamLegacy &&
+                      stream != cudaStreamPerThread;
+  if (!usable) return encode_impl(e, in, workspace, workspace_bytes, cu_dev, sm_budget, stream_v, out_embeddings);
+  const int n = in->n_items;
+  std::vector<int64_t> key;
+  key.reserve(8 + 5 * static_cast<size_t>(n) + 1);
+  key.push_back(n); key.push_back(sm_budget); key.push_back(e->attn_impl);
+  key.push_back(static_cast<int64_t>(reinterpret_cast<uintptr_t>(in->data)));
+  key.push_back(static_cast<int64_t>(reinterpret_cast<uintptr_t>(workspace)));
+  key.push_back(static_cast<int64_t>(workspace_bytes));
+  key.push_back(static_cast<int64_t>(reinterpret_cast<uintptr_t>(cu_dev)));
+  key.push_back(static_cast<int64_t>(reinterpret_cast<uintptr_t>(out_embeddings)));
+  for (int i = 0; i < 3 * n; ++i) key.push_back(in->item_shape[i]);
+  for (int i = 0; i < n; ++i) key.push_back(in->item_offset[i]);
+  for (int i = 0; i <= n; ++i) key.push_back(in->cu_seqlens_host[i]);
+  ++e->graph_clock;
+  for (GraphEntry& g : e->graphs) {
+    if (g.key == key) {
+      g.last_use = e->graph_clock;
+      e->last_launches = g.launches;
+      e->last_status = g.status;
+      ++e->graph_hits;
+      CUDA_TRY(cudaGraphLaunch(g.exec, stream));
+      return EAS_OK;
+    }
+  }
+  cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+  CUDA_TRY(cudaStreamIsCapturing(stream, &cap));
+  if (cap != cudaStreamCaptureStatusNone)     // the caller is capturing this stream itself: just add the launches
+    return encode_impl(e, in, workspace, workspace_bytes, cu_dev, sm_budget, stream_v, out_embeddings);
+  CUDA_TRY(cudaStreamBeginCapture(stream, cudaStreamCaptureModeRelaxed));
+  const eas_status st = encode_impl(e, in, workspace, workspace_bytes, cu_dev, sm_budget, stream_v, out_embeddings);
+  cudaGraph_t graph = nullptr;
+  const cudaError_t end = cudaStreamEndCapture(stream, &graph);
+  if (st != EAS_OK) {                         // nothing was launched; the message of the failed step stands
+    if (graph) cudaGraphDestroy(graph);
+    (void)cudaGetLastError();
+    return st;
+  }
+  if (end != cudaSuccess || graph == nullptr) {
+    if (graph) cudaGraphDestroy(graph);
+    return fail(EAS_ERR_CUDA, "stream capture of the forward pass failed: %s", cudaGetErrorString(end));
+  }
+  GraphEntry g;
+  const cudaError_t inst = cudaGraphInstantiate(&g.exec, graph, 0);
+  cudaGraphDestroy(graph);
+  if (inst != cudaSuccess) return fail(EAS_ERR_CUDA, "cudaGraphInstantiate failed: %s", cudaGetErrorString(inst));
+  g.key = std::move(key);
+  g.launches = e->last_launches;
+  g.status = e->last_status;
+  g.last_use = e->graph_clock;
+  if (e->graphs.size() >= kMaxGraphs) {       // evict the least recently used capture
+    size_t victim = 0;
+    for (size_t i = 1; i < e->graphs.size(); ++i) if (e->graphs[i].last_use < e->graphs[victim].last_use) victim = i;
+    cudaGraphExecDestroy(e->graphs[victim].exec);
+    e->graphs[victim] = std::move(g);
+    ++e->graph_captures;
+    CUDA_TRY(cudaGraphLaunch(e->graphs[victim].exec, stream));
+    return EAS_OK;
+  }
+  e->graphs.push_back(std::move(g));
+  ++e->graph_captures;
+  CUDA_TRY(cudaGraphLaunch(e->graphs.back().exec, stream));
+  return EAS_OK;
+}
+
 extern "C" eas_status eas_encode_microbatch(eas_encoder* e, const eas_packed_inputs* in, const int32_t* cu_dev,
                                             int32_t sm_budget, void* stream_v, void* out_embeddings) {
   if (in == nullptr) return fail(EAS_ERR_INVALID_ARG, "encoder or inputs are null");
-  return encode_impl(e, in, in->workspace, in->workspace_bytes, cu_dev, sm_budget, stream_v, out_embeddings);
+  return encode_cached(e, in, in->workspace, in->workspace_bytes, cu_dev, sm_budget, stream_v, out_embeddings);
+}
+
+extern "C" eas_status eas_encoder_set_graph_mode(eas_encoder* e, int32_t mode) {
+  if (e == nullptr) return fail(EAS_ERR_INVALID_ARG, "encoder is null");
+  if (mode != 0 && mode != 1) return fail(EAS_ERR_INVALID_ARG, "graph mode %d (0 = off, 1 = on)", mode);
+  e->graph_mode = mode;
+  if (mode == 0) {
+    for (GraphEntry& g : e->graphs) if (g.exec) cudaGraphExecDestroy(g.exec);
+    e->graphs.clear();
+  }
+  return EAS_OK;
+}
+
+extern "C" eas_status eas_encoder_graph_stats(const eas_encoder* e, int64_t* hits, int64_t* captures, int32_t* cached) {
+  if (e == nullptr) return fail(EAS_ERR_INVALID_ARG, "encoder is null");
+  if (hits) *hits = e->graph_hits;
+  if (captures) *captures = e->graph_captures;
+  if (cached) *cached = static_cast<int32_t>(e->graphs.size());
+  return EAS_OK;
 }
 
 // ------------------------------------------------------------------------------------ scratch baked into the library
@@ -983,7 +1093,7 @@ extern "C" eas_status eas_encode_microbatch_static(eas_encoder* e, const eas_pac
                     "with a caller-allocated workspace, or send fewer / smaller items", need, usable);
     }
   }
-  return encode_impl(e, in, reinterpret_cast<void*>(aligned), usable, cu_dev, sm_budget, stream_v, out_embeddings);
+  return encode_cached(e, in, reinterpret_cast<void*>(aligned), usable, cu_dev, sm_budget, stream_v, out_embeddings);
 }
 
 extern "C" eas_status eas_encoder_enable_timing(eas_encoder* e, int32_t on) {
