@@ -63,6 +63,16 @@ int32_t eas_router_next(eas_router* r);                                         
 int32_t eas_envelope_plan(const int32_t* dest, const int32_t* rows, int32_t n_requests, int32_t n_dest,
                           int64_t* row_offset, int64_t* dest_rows);
 
+/* Encode order that lays the envelopes out back to back in the encoder's output.  The encoder writes the embedding rows
+ * of its items in the order the items are listed, and items do not interact (block-diagonal attention), so listing the
+ * requests of a micro-batch grouped by destination makes the final epilogue itself write every request into its
+ * destination's contiguous envelope: no gather after the forward pass.  order[k] receives the index of the request to list
+ * k-th (a stable sort by destination, so arrival order is kept inside an envelope, as in eas_envelope_plan);
+ * env_first_row[d] receives the first output row of destination d's envelope.  Request i then occupies rows
+ * [env_first_row[dest[i]] + row_offset[i], + rows[i]) of out_embeddings.  Returns 0, or -1 on a bad argument. */
+int32_t eas_envelope_order(const int32_t* dest, const int32_t* rows, int32_t n_requests, int32_t n_dest, int32_t* order,
+                           int64_t* env_first_row);
+
 /* ---- Section 3.4: SM lookup table ---------------------------------------------------------------------------------- */
 
 enum { EAS_SM_TABLE_MAX_LEVELS = 16 };

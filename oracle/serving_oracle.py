@@ -62,6 +62,17 @@ def envelope_plan(dest, rows, n_dest):
     return offs, totals
 
 
+def envelope_order(dest, rows, n_dest):
+    """Section 3.3: the order of requests that makes each destination's envelope one contiguous block of the output
+    (stable by destination), and the first output row of each envelope."""
+    order = sorted(range(len(dest)), key=lambda i: dest[i])          # Python's sort is stable
+    first, acc = [], 0
+    for d in range(n_dest):
+        first.append(acc)
+        acc += sum(r for dd, r in zip(dest, rows) if dd == d)
+    return order, first
+
+
 def sm_table_build(sm_counts, batches, latency, exclusive, tol=0.2):
     """Section 3.4: per SM level, the largest profiled batch size whose latency stays within (1 + tol) of exclusive
     access (reading: all smaller profiled sizes must hold too)."""

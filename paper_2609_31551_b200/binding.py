@@ -268,14 +268,16 @@ class Encoder:
         return self.lib.eas_encoder_last_launch_count(self.handle)
 
 
-def kernel_gemm(A, W, bias, act=0, out_fp32=False, resid=None, sm_budget=0, stream=None, out=None):
-    """eas_kernel_gemm on device tensors.  Returns out."""
+def kernel_gemm(A, W, bias, act=0, out_fp32=False, resid=None, sm_budget=0, stream=None, out=None, status=None):
+    """eas_kernel_gemm on device tensors.  Returns (out, device status word).  `status` (device int32, zeroed by the
+    caller) can be passed in so that a call allocates nothing."""
     lib = load_library()
     M, K = A.shape
     N = W.shape[0]
     if out is None:
         out = torch.empty((M, N // 2 if act == 2 else N), dtype=torch.float32 if out_fp32 else torch.bfloat16, device=A.device)
-    status = torch.zeros(4, dtype=torch.int32, device=A.device)
+    if status is None:
+        status = torch.zeros(4, dtype=torch.int32, device=A.device)
     _check(lib.eas_kernel_gemm(A.data_ptr(), W.data_ptr(), bias.data_ptr(), out.data_ptr(),
                                resid.data_ptr() if resid is not None else None, M, N, K, act, int(out_fp32), sm_budget,
                                _stream_ptr(stream), status.data_ptr()))

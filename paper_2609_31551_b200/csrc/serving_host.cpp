@@ -113,6 +113,26 @@ extern "C" int32_t eas_envelope_plan(const int32_t* dest, const int32_t* rows, i
   return 0;
 }
 
+extern "C" int32_t eas_envelope_order(const int32_t* dest, const int32_t* rows, int32_t n, int32_t n_dest, int32_t* order,
+                                      int64_t* env_first_row) {
+  if (dest == nullptr || rows == nullptr || order == nullptr || env_first_row == nullptr || n < 0 || n_dest <= 0) return -1;
+  // counting sort by destination (stable: arrival order is kept inside an envelope)
+  std::vector<int64_t> count(static_cast<size_t>(n_dest) + 1, 0), total(static_cast<size_t>(n_dest), 0);
+  for (int32_t i = 0; i < n; ++i) {
+    if (dest[i] < 0 || dest[i] >= n_dest || rows[i] < 0) return -1;
+    ++count[static_cast<size_t>(dest[i]) + 1];
+    total[static_cast<size_t>(dest[i])] += rows[i];
+  }
+  int64_t first = 0;
+  for (int32_t k = 0; k < n_dest; ++k) {
+    count[static_cast<size_t>(k) + 1] += count[static_cast<size_t>(k)];
+    env_first_row[k] = first;
+    first += total[static_cast<size_t>(k)];
+  }
+  for (int32_t i = 0; i < n; ++i) order[count[static_cast<size_t>(dest[i])]++] = i;
+  return 0;
+}
+
 // ------------------------------------------------------------------------------------ SM lookup table
 extern "C" int32_t eas_sm_table_build(const int32_t* sm_counts, int32_t n_levels, const int32_t* batches, int32_t n_batches,
                                       const double* latency, const double* exclusive, double tolerance, eas_sm_table* out) {

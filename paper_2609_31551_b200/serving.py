@@ -7,7 +7,7 @@ from .binding import load_library
 SERVING_SYMBOLS = [
     "eas_poisson_gap_kappa", "eas_batcher_create", "eas_batcher_destroy", "eas_batcher_gap", "eas_batcher_deadline",
     "eas_batcher_on_arrival", "eas_batcher_on_timer", "eas_router_init", "eas_router_init_from_double", "eas_router_next",
-    "eas_envelope_plan", "eas_sm_table_build", "eas_sm_table_lookup", "eas_has_stage1",
+    "eas_envelope_plan", "eas_envelope_order", "eas_sm_table_build", "eas_sm_table_lookup", "eas_has_stage1",
 ]
 
 
@@ -55,6 +55,9 @@ def lib():
         l.eas_envelope_plan.restype = C.c_int32
         l.eas_envelope_plan.argtypes = [C.POINTER(C.c_int32), C.POINTER(C.c_int32), C.c_int32, C.c_int32,
                                         C.POINTER(C.c_int64), C.POINTER(C.c_int64)]
+        l.eas_envelope_order.restype = C.c_int32
+        l.eas_envelope_order.argtypes = [C.POINTER(C.c_int32), C.POINTER(C.c_int32), C.c_int32, C.c_int32,
+                                         C.POINTER(C.c_int32), C.POINTER(C.c_int64)]
         l.eas_sm_table_build.restype = C.c_int32
         l.eas_sm_table_build.argtypes = [C.POINTER(C.c_int32), C.c_int32, C.POINTER(C.c_int32), C.c_int32,
                                          C.POINTER(C.c_double), C.POINTER(C.c_double), C.c_double, C.POINTER(SmTable)]
@@ -119,6 +122,19 @@ def envelope_plan(dest, rows, n_dest):
     if rc != 0:
         raise ValueError("bad envelope arguments")
     return offs.tolist(), tot.tolist()
+
+
+def envelope_order(dest, rows, n_dest):
+    """eas_envelope_order -> (order of the requests that groups them by destination, first output row per envelope)."""
+    d = np.ascontiguousarray(dest, dtype=np.int32)
+    r = np.ascontiguousarray(rows, dtype=np.int32)
+    order = np.zeros(len(d), dtype=np.int32)
+    first = np.zeros(n_dest, dtype=np.int64)
+    rc = lib().eas_envelope_order(d.ctypes.data_as(C.POINTER(C.c_int32)), r.ctypes.data_as(C.POINTER(C.c_int32)), len(d), n_dest,
+                                  order.ctypes.data_as(C.POINTER(C.c_int32)), first.ctypes.data_as(C.POINTER(C.c_int64)))
+    if rc != 0:
+        raise ValueError("bad envelope arguments")
+    return order.tolist(), first.tolist()
 
 
 def sm_table_build(sm_counts, batches, latency, exclusive, tol=0.2) -> SmTable:

@@ -2,6 +2,9 @@
 latency sweep, and a simulated arrival trace through batcher -> SM lookup -> encode -> router/envelopes."""
 import numpy as np
 import pytest
+import torch
+
+import eas_synth as S
 
 pytestmark = pytest.mark.gpu
 
@@ -23,3 +26,47 @@ def test_profiling_and_simulated_serving_on_c0():
     assert abs(res["remote_fraction"] - 0.7) < 0.01                               # the router holds the ratio
     assert res["transfers"] <= 3 * res["dispatches"]                              # at most one envelope per destination
     assert res["encode_latency_p99_s"] < 1.0 + 0.5                                # the age cap bounds the wait
+
+
+def test_grouped_item_order_writes_each_request_into_its_envelope():
+    """Section 3.3: with the requests listed in eas_envelope_order's order, the forward pass itself writes every
+    request's embeddings into its destination's contiguous envelope, bit-identical to encoding in arrival order."""
+    import paper_2609_31551_b200 as P
+    from paper_2609_31551_b200 import serving as SV
+    cfg = S.get_config("c2")
+    enc = P.Encoder(cfg, P.weights_to_device(S.make_weights(cfg)))
+    shapes = [(1, 224, 280), (1, 336, 224), (1, 224, 224), (1, 280, 280), (1, 224, 336)]
+    dest = [1, 0, 2, 0, 1]
+    items = S.make_items(cfg, shapes, seed=31)
+    data, offsets = P.pack_items(items)
+    tok = [S.tokens_per_item(cfg, s) for s in shapes]
+    rows = [S.out_tokens_per_item(cfg, s) for s in shapes]
+    cu = np.concatenate([[0], np.cumsum(tok)]).astype(np.int32)
+    ref = enc.encode_microbatch(data, shapes, offsets, cu)
+    enc.status()
+    order, first = SV.envelope_order(dest, rows, 3)
+    offs, totals = SV.envelope_plan(dest, rows, 3)
+    g_shapes = [shapes[i] for i in order]
+    g_offsets = [offsets[i] for i in order]             # the items stay where they are in `data`: only the listing changes
+    g_cu = np.concatenate([[0], np.cumsum([tok[i] for i in order])]).astype(np.int32)
+    out = enc.encode_microbatch(data, g_shapes, g_offsets, g_cu)
+    enc.status()
+    ref_start = np.concatenate([[0], np.cumsum(rows)])
+    for i in range(len(shapes)):
+        lo = first[dest[i]] + offs[i]
+        assert torch.equal(out[lo: lo + rows[i]], ref[ref_start[i]: ref_start[i] + rows[i]]), f"request {i}"
+    assert sum(totals) == out.shape[0]
+
+
+def test_coresidency_measurement_runs_and_reports_sane_numbers():
+    """Encoder on a share of the SMs beside a GEMM stream on the rest (Section 3.4): structural checks only, the
+    figures themselves are machine-dependent."""
+    from paper_2609_31551_b200 import coresidency as CR
+    rows = CR.measure("c0", 4, levels=(0.5,), reps=3, neighbour_shape=(2048, 2048, 2048))
+    assert len(rows) == 1
+    r = rows[0]
+    assert r["sm_encode"] + r["sm_neighbour"] == torch.cuda.get_device_properties(0).multi_processor_count
+    for k in ("encode_ms_exclusive", "encode_ms_alone", "encode_ms_beside_neighbour", "neighbour_tflops_alone",
+              "neighbour_tflops_beside_encoder"):
+        assert np.isfinite(r[k]) and r[k] > 0
+    assert 0.5 < r["inflation"] < 20

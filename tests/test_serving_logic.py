@@ -140,6 +140,10 @@ def test_library_router_envelopes_and_table_match_oracle(sv):
     assert sv.envelope_plan(dest, rows, 3) == tuple(SO.envelope_plan(dest, rows, 3))
     with pytest.raises(ValueError):
         sv.envelope_plan([0, 5], [1, 1], 3)
+    assert sv.envelope_order(dest, rows, 3) == tuple(SO.envelope_order(dest, rows, 3))
+    assert sv.envelope_order([], [], 2) == ([], [0, 0])
+    with pytest.raises(ValueError):
+        sv.envelope_order([0, 3], [1, 1], 3)
     levels, batches = [15, 44, 74, 104, 133], [1, 2, 4, 8, 16]
     lat = rng.uniform(1.0, 2.0, size=(5, 5)) * np.array([[1, 2, 4, 8, 16]])
     excl = np.array([1.0, 2.0, 4.0, 8.0, 16.0]) * 1.1
@@ -173,3 +177,27 @@ def test_has_stage1_oracle_properties_and_library(sv):
     assert sv.has_stage1(cands, 500.0, cE, cP, cD, alpha)[1] == []
     with pytest.raises(ValueError):
         sv.has_stage1([(0, 1, 1, 0)], rate, cE, cP, cD, alpha)
+
+
+def test_envelope_order_lays_envelopes_out_back_to_back():
+    """Pin of the oracle by construction: write each request's rows in the returned order into one buffer and check
+    that every destination's rows form one contiguous block, in arrival order, at the offsets of the envelope plan."""
+    rng = np.random.Generator(np.random.PCG64(11))
+    for n, n_dest in ((1, 1), (7, 3), (40, 4), (64, 2)):
+        dest = rng.integers(0, n_dest, size=n).tolist()
+        rows = rng.integers(1, 50, size=n).tolist()
+        order, first = SO.envelope_order(dest, rows, n_dest)
+        offs, totals = SO.envelope_plan(dest, rows, n_dest)
+        assert sorted(order) == list(range(n))
+        owner = []                                   # request id of every output row, in encode order
+        for i in order:
+            owner += [i] * rows[i]
+        for d in range(n_dest):
+            block = owner[first[d]: first[d] + totals[d]]
+            expect = []
+            for i in range(n):
+                if dest[i] == d:
+                    assert owner.index(i) == first[d] + offs[i] if rows[i] else True
+                    expect += [i] * rows[i]
+            assert block == expect
+        assert first[0] == 0 and all(first[d + 1] == first[d] + totals[d] for d in range(n_dest - 1))
