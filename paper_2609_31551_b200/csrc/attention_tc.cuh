@@ -3,6 +3,9 @@
 // One work unit = (item, head, 256 query rows) = two 128-row query tiles A and B that share every
 // K/V tile.  Keys and values come from the same item only: the key loop stops at the item's last
 // 128-key tile and the keys past the item's end are masked to -inf (probability exactly 0).
+// An item with an odd number of query tiles (577 tokens = 4.5 tiles) would leave tile B empty in every
+// head's last unit; for head_dim 64 those last tiles of two adjacent heads share a unit instead
+// (dual-head unit: A on head h, B on head h + 1, each with its own K/V tiles).
 //
 //   warp 0       TMA producer: Q tiles (double buffered across units), K/V tiles through a ring
 //   warp 1       UMMA issuer:  S = Q K^T (128x128x{64|80}) into TMEM, O += P V (128x{64|80}x128) in TMEM
@@ -66,6 +69,11 @@ struct AttnTcSmem {
   // TMEM columns: S_A [0,128) S_B [128,256) O_A [256,256+HD) O_B [256+HD', ...).  P in tensor memory: head_dim 64 has
   // room for dedicated columns; head_dim 80 re-uses the first 64 columns of S (dead once the row sits in registers),
   // which obliges the issuer to run P V before the next S.
+  // Dual-head units: an item whose query rows end in a single 128-row tile would leave warpgroup B idle for that
+  // tile's whole key loop (c1: 577 tokens = 4.5 tiles, one unit in three).  With four K/V stages such tiles of TWO
+  // adjacent heads form one unit instead: A works on head h, B on head h + 1, each with its own K/V tiles (two ring
+  // stages per key tile).
+  static constexpr bool kDualHeadOk = PT && HD == 64;   // the kernel's DUAL template argument may be set
   static constexpr int kOCol0 = 256, kOStride = HD == 64 ? 64 : 128;
   static constexpr bool kPAliasesS = PT && HD != 64;
   static constexpr int kPCol0 = kPAliasesS ? 0 : 384, kPStride = kPAliasesS ? 128 : 64;
@@ -166,10 +174,15 @@ __device__ unsigned long long g_attn_dbg[2 * 64 * 12];
 
 struct UnitInfo {
   int head, q0, S, n_kv, n_q;
+  int dual;             // 1: tile A belongs to `head`, tile B to `head + 1`, same query rows, separate K/V tiles
   long long row0;
 };
 // `cursor` is the caller's item index of its previous unit: units are visited in increasing order, so the item is
 // found by stepping forward (usually zero or one step) instead of searching.
+// Unit order inside an item (the host's attention_schedule counts the same way).  Without dual-head units:
+// (head, pair of query tiles), the pair index fastest, the last pair possibly a single tile.  With them: first the
+// (head, FULL pair) units, then one unit per two heads for the odd last query tile.
+template <bool DUAL>
 __device__ __forceinline__ UnitInfo decode_unit(const AttnTcParams& p, int unit, int& cursor) {
   int lo = cursor;
   while (lo + 1 < p.n_items && p.unit_prefix[lo + 1] <= unit) ++lo;
@@ -177,18 +190,38 @@ __device__ __forceinline__ UnitInfo decode_unit(const AttnTcParams& p, int unit,
   UnitInfo u;
   u.S = p.item_len[lo];
   u.row0 = p.item_start[lo];
-  const int pairs = (u.S + 2 * kTcTile - 1) / (2 * kTcTile);
+  u.n_kv = (u.S + kTcTile - 1) / kTcTile;
   const int r = unit - p.unit_prefix[lo];
+  if (DUAL) {
+    const int full = u.n_kv >> 1;                  // query tiles == key tiles
+    const int n_full = p.n_heads * full;
+    if (r < n_full) {
+      u.head = r / full;
+      u.q0 = (r - u.head * full) * 2 * kTcTile;
+      u.n_q = 2;
+      u.dual = 0;
+    } else {
+      u.head = 2 * (r - n_full);
+      u.q0 = full * 2 * kTcTile;
+      u.dual = u.head + 1 < p.n_heads ? 1 : 0;
+      u.n_q = 1 + u.dual;
+    }
+    return u;
+  }
+  const int pairs = (u.S + 2 * kTcTile - 1) / (2 * kTcTile);
   u.head = r / pairs;
   u.q0 = (r - u.head * pairs) * 2 * kTcTile;       // pair index varies fastest: neighbours share K and V in L2
-  u.n_kv = (u.S + kTcTile - 1) / kTcTile;
   u.n_q = (u.q0 + kTcTile < u.S) ? 2 : 1;
+  u.dual = 0;
   return u;
 }
 
-template <int HD, bool PT>
+// DUAL: the launch's unit order contains dual-head units (the host sets it only when some item has an odd number of
+// query tiles; without it every `dual` test below folds away).
+template <int HD, bool PT, bool DUAL = false>
 __global__ void __launch_bounds__(kTcThreads, 1) attn_tc_kernel(const __grid_constant__ AttnTcParams p) {
   using L = AttnTcSmem<HD, PT>;
+  static_assert(!DUAL || L::kDualHeadOk, "dual-head units need four K/V stages and dedicated P columns");
   constexpr int HI = L::HI;
   constexpr int NST = L::kStages;
   extern __shared__ uint8_t smem_raw_attn[];
@@ -242,17 +275,20 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_tc_kernel(const __grid_con
       bool ok = true;
       int cursor = 0;
       for (int unit = blockIdx.x; unit < p.total_units && ok; unit += gridDim.x, ++u_cnt) {
-        const UnitInfo u = decode_unit(p, unit, cursor);
+        const UnitInfo u = decode_unit<DUAL>(p, unit, cursor);
         const int qb = u_cnt & 1;
         if (!mbar_wait(&q_empty[qb], ((u_cnt >> 1) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
         mbar_expect_tx(&q_full[qb], u.n_q * L::kTileBytes);
-        const int xq = u.head * HD;
         for (int t = 0; t < u.n_q; ++t) {
-          const int y = static_cast<int>(u.row0) + u.q0 + t * kTcTile;
+          const int xq = (u.head + (u.dual ? t : 0)) * HD;
+          const int y = static_cast<int>(u.row0) + u.q0 + (u.dual ? 0 : t * kTcTile);
           tma_load_2d(q_tile(qb, t), &p.map_lo, &q_full[qb], xq, y);
           if (HI) tma_load_2d(q_tile(qb, t) + L::kLoBytes, &p.map_hi, &q_full[qb], xq + 64, y);
         }
-        for (int j = 0; j < u.n_kv; ++j, ++kv_it) {
+        const int kv_tiles = u.n_kv * (1 + u.dual);      // dual-head units: key tile j of head h, then of head h + 1
+        for (int jj = 0; jj < kv_tiles; ++jj, ++kv_it) {
+          const int j = u.dual ? (jj >> 1) : jj;
+          const int xq = (u.head + (u.dual ? (jj & 1) : 0)) * HD;
           const int s = kv_it % NST;
           if (!mbar_wait(&kv_empty[s], ((kv_it / NST) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
           const int y = static_cast<int>(u.row0) + j * kTcTile;
@@ -334,29 +370,39 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_tc_kernel(const __grid_con
 
       bool pre_issued[2] = {false, false};       // S(w, 0) of this unit was already issued at the end of the previous one
       int cursor = 0;
-      UnitInfo un = decode_unit(p, min(static_cast<int>(blockIdx.x), p.total_units - 1), cursor);
+      UnitInfo un = decode_unit<DUAL>(p, min(static_cast<int>(blockIdx.x), p.total_units - 1), cursor);
       for (int unit = blockIdx.x; unit < p.total_units && ok; unit += gridDim.x, ++u_cnt) {
         const UnitInfo u = un;
         const int qb = u_cnt & 1;
         const bool has_next = unit + static_cast<int>(gridDim.x) < p.total_units;
-        if (has_next) un = decode_unit(p, unit + gridDim.x, cursor);
+        if (has_next) un = decode_unit<DUAL>(p, unit + gridDim.x, cursor);
         if (!mbar_wait(&q_full[qb], (u_cnt >> 1) & 1u, abort_flag)) { ok = false; break; }
-        {
-          const int s = kv_it % NST;
-          if (!mbar_wait(&k_full[s], (kv_it / NST) & 1u, abort_flag)) { ok = false; break; }
-          tc_fence_after_sync();
+        // K/V tile of warpgroup w at ring position kv_it: shared by both warpgroups, or (dual-head unit) one each
+        const uint32_t step = 1 + u.dual;
 #pragma unroll
-          for (int w = 0; w < 2; ++w) if (w < u.n_q && !pre_issued[w]) issue_s(w, qb, s);
-          pre_issued[0] = pre_issued[1] = false;
+        for (int w = 0; w < 2; ++w) {
+          if (w < u.n_q && !pre_issued[w]) {
+            const uint32_t g = kv_it + (u.dual ? w : 0);
+            if (!mbar_wait(&k_full[g % NST], (g / NST) & 1u, abort_flag)) { ok = false; break; }
+            tc_fence_after_sync();
+            issue_s(w, qb, g % NST);
+          }
         }
+        if (!ok) break;
+        pre_issued[0] = pre_issued[1] = false;
         bool next_q_ready = false;
-        for (int j = 0; j < u.n_kv && ok; ++j, ++kv_it) {
-          const int s = kv_it % NST;
-          const int sn = (kv_it + 1) % NST;
-          const bool last = j + 1 == u.n_kv;
+        const int n_kv = u.n_kv, n_q = u.n_q, next_n_q = un.n_q;
+        const uint32_t b_off = u.dual ? 1u : 0u, b_off_next = un.dual ? 1u : 0u;   // B's tile relative to A's
+        for (int j = 0; j < n_kv && ok; ++j, kv_it += step) {
+          const bool last = j + 1 == n_kv;
 #pragma unroll
           for (int w = 0; w < 2; ++w) {
-            if (w >= u.n_q) break;
+            if (w >= n_q) break;
+            const uint32_t g = kv_it + (w ? b_off : 0u);                                          // this tile
+            const uint32_t gn = kv_it + step + (w ? (last ? b_off_next : b_off) : 0u);            // the warpgroup's next one
+            const int s = g % NST, sn = gn % NST;
+            // warpgroup B shares A's tiles unless the unit is dual-head: A has already seen them land
+            const bool own_tile = w == 0 || (b_off | (last ? b_off_next : 0u)) != 0u;
             // P(w, j) is in shared memory, S(w) has been read, O(w) has been rescaled if it had to be
             if (!mbar_wait(&p_ready[w], (n_pv[w]) & 1u, abort_flag)) { ok = false; break; }
             tc_fence_after_sync();
@@ -364,31 +410,33 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_tc_kernel(const __grid_con
             // tile the next scores are the first tile of the NEXT unit, so the pipeline never drains
             // next scores before P V, so that the next softmax overlaps it -- unless P re-uses S's columns
             if (!last && !L::kPAliasesS) {
-              if (w == 0 && !mbar_wait(&k_full[sn], ((kv_it + 1) / NST) & 1u, abort_flag)) { ok = false; break; }
+              if (own_tile && !mbar_wait(&k_full[sn], (gn / NST) & 1u, abort_flag)) { ok = false; break; }
               tc_fence_after_sync();
               issue_s(w, qb, sn);
             }
-            if (w == 0 && !mbar_wait(&v_full[s], (kv_it / NST) & 1u, abort_flag)) { ok = false; break; }
+            if (own_tile && !mbar_wait(&v_full[s], (g / NST) & 1u, abort_flag)) { ok = false; break; }
             tc_fence_after_sync();
             issue_pv(w, s, j != 0);
             if (!last && L::kPAliasesS) {
-              if (w == 0 && !mbar_wait(&k_full[sn], ((kv_it + 1) / NST) & 1u, abort_flag)) { ok = false; break; }
+              if (own_tile && !mbar_wait(&k_full[sn], (gn / NST) & 1u, abort_flag)) { ok = false; break; }
               tc_fence_after_sync();
               issue_s(w, qb, sn);
             }
-            if (last && has_next && w < un.n_q) {
+            if (last && has_next && w < next_n_q) {
               // the unit's output is waiting for this P V, so it went first; now the first scores of the next unit
               if (!next_q_ready) {
                 if (!mbar_wait(&q_full[qb ^ 1], ((u_cnt + 1) >> 1) & 1u, abort_flag)) { ok = false; break; }
                 next_q_ready = true;
               }
-              if (w == 0 && !mbar_wait(&k_full[sn], ((kv_it + 1) / NST) & 1u, abort_flag)) { ok = false; break; }
+              if (own_tile && !mbar_wait(&k_full[sn], (gn / NST) & 1u, abort_flag)) { ok = false; break; }
               tc_fence_after_sync();
               issue_s(w, qb ^ 1, sn);
               pre_issued[w] = true;
             }
+            // K and V of this tile are free once everything issued so far completes: after the last warpgroup that
+            // uses them
+            if (b_off != 0u || w + 1 == n_q) umma_commit(&kv_empty[s]);
           }
-          if (ok) umma_commit(&kv_empty[s]);   // K(j) and V(j) are free once everything issued so far completes
         }
         if (ok) umma_commit(&q_empty[qb]);
       }
@@ -423,7 +471,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_tc_kernel(const __grid_con
       tc_fence_after_sync();
       ATTN_STAMP_PREV(7);
       const float inv = 1.0f / pend_l;
-      const int warp_row0 = pend_q0 + w * kTcTile + quarter * 32;      // first query row of this warp within the item
+      const int warp_row0 = pend_q0 + quarter * 32;                    // first query row of this warp within the item
       const int qrow = warp_row0 + lane;
       uint32_t o[HD / 16][16];
       __syncwarp();
@@ -467,13 +515,13 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_tc_kernel(const __grid_con
     };
 
     int cursor = 0;
-    UnitInfo u_next = decode_unit(p, min(static_cast<int>(blockIdx.x), p.total_units - 1), cursor);
+    UnitInfo u_next = decode_unit<DUAL>(p, min(static_cast<int>(blockIdx.x), p.total_units - 1), cursor);
     for (int unit = blockIdx.x; unit < p.total_units && ok; unit += gridDim.x) {
       const UnitInfo u = u_next;
       ATTN_STAMP_PREV(10);
       const bool has_next = unit + static_cast<int>(gridDim.x) < p.total_units;
       if (w >= u.n_q) {                             // this warpgroup has no tile in the unit
-        if (has_next) u_next = decode_unit(p, unit + gridDim.x, cursor);
+        if (has_next) u_next = decode_unit<DUAL>(p, unit + gridDim.x, cursor);
         if (pend && !flush_output()) { ok = false; break; }
         continue;
       }
@@ -593,11 +641,13 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_tc_kernel(const __grid_con
         if (lane == 0) mbar_arrive(&p_ready[w]);
         ATTN_STAMP(6);
         // decode the following unit here: the warp now waits for the issuer anyway
-        if (j == 0 && has_next) u_next = decode_unit(p, unit + gridDim.x, cursor);
+        if (j == 0 && has_next) u_next = decode_unit<DUAL>(p, unit + gridDim.x, cursor);
       }
       if (!ok) break;
       pend = true;                                  // written later, see flush_output
-      pend_q0 = u.q0; pend_head = u.head; pend_S = u.S; pend_row0 = u.row0; pend_l = l; pend_n = n - 1;
+      // this warpgroup's tile: the second 128 rows of the same head, or (dual-head unit) the same rows of the next head
+      pend_q0 = u.q0 + (u.dual ? 0 : w * kTcTile); pend_head = u.head + (u.dual ? w : 0);
+      pend_S = u.S; pend_row0 = u.row0; pend_l = l; pend_n = n - 1;
     }
     if (ok && pend) flush_output();
     if (L::kStagedOut && lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");

@@ -636,8 +636,10 @@ static eas_status launch_norm(int kind, bool out_fp32, const NormParams& p, int 
 }
 
 // schedule order: longest items first (stable), so the tail of the static round-robin is short work
+// dual_head: the tcgen05 kernel's unit order for head_dim 64 (see decode_unit): per item H x (full pairs of query
+// tiles), then one unit per two heads for an odd last tile.
 static void attention_schedule(const int32_t* cu, int n_items, int rows_per_unit, int H, int* item_start, int* item_len,
-                               int* unit_prefix, int* total_units) {
+                               int* unit_prefix, int* total_units, bool dual_head = false) {
   std::vector<int> order(n_items);
   for (int i = 0; i < n_items; ++i) order[i] = i;
   std::stable_sort(order.begin(), order.end(), [&](int a, int b) { return (cu[a + 1] - cu[a]) > (cu[b + 1] - cu[b]); });
@@ -647,7 +649,12 @@ static void attention_schedule(const int32_t* cu, int n_items, int rows_per_unit
     item_start[k] = cu[i];
     item_len[k] = cu[i + 1] - cu[i];
     unit_prefix[k] = units;
-    units += ((item_len[k] + rows_per_unit - 1) / rows_per_unit) * H;
+    if (dual_head) {
+      const int tiles = (item_len[k] + rows_per_unit / 2 - 1) / (rows_per_unit / 2);
+      units += (tiles / 2) * H + (tiles % 2) * ((H + 1) / 2);
+    } else {
+      units += ((item_len[k] + rows_per_unit - 1) / rows_per_unit) * H;
+    }
   }
   unit_prefix[n_items] = units;
   *total_units = units;
@@ -697,15 +704,23 @@ static eas_status launch_attention_tc(const bf16* qkv, bf16* out, const int32_t*
   ap.scale_log2 = static_cast<float>(1.4426950408889634 / std::sqrt(static_cast<double>(hd)));
   ap.n_items = n_items;
   ap.status = status;
-  attention_schedule(cu, n_items, 2 * kTcTile, H, ap.item_start, ap.item_len, ap.unit_prefix, &ap.total_units);
+  // dual-head units (two heads' odd last query tiles in one unit) when some item has an odd number of 128-row tiles
+  bool dual = false;
+  if (hd == 64 && AttnTcSmem<64, PT>::kDualHeadOk && H >= 2)
+    for (int i = 0; i < n_items; ++i) dual = dual || (((cu[i + 1] - cu[i] + kTcTile - 1) / kTcTile) & 1) != 0;
+  attention_schedule(cu, n_items, 2 * kTcTile, H, ap.item_start, ap.item_len, ap.unit_prefix, &ap.total_units, dual);
   if (ap.total_units == 0) return EAS_OK;
   const int grid = std::min(budget, ap.total_units);
   static bool attr_set = false;
   if (!attr_set) {
     CUDA_TRY(cudaFuncSetAttribute(attn_tc_kernel<64, PT>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttnTcSmem<64, PT>::kBytes));
     CUDA_TRY(cudaFuncSetAttribute(attn_tc_kernel<80, PT>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttnTcSmem<80, PT>::kBytes));
+    if (AttnTcSmem<64, PT>::kDualHeadOk)
+      CUDA_TRY(cudaFuncSetAttribute(attn_tc_kernel<64, PT, AttnTcSmem<64, PT>::kDualHeadOk>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttnTcSmem<64, PT>::kBytes));
     attr_set = true;
   }
+  if (hd == 64 && dual)
+    return launch_kernel(attn_tc_kernel<64, PT, AttnTcSmem<64, PT>::kDualHeadOk>, grid, kTcThreads, AttnTcSmem<64, PT>::kBytes, stream, ap);
   if (hd == 64) return launch_kernel(attn_tc_kernel<64, PT>, grid, kTcThreads, AttnTcSmem<64, PT>::kBytes, stream, ap);
   if (hd == 80) return launch_kernel(attn_tc_kernel<80, PT>, grid, kTcThreads, AttnTcSmem<80, PT>::kBytes, stream, ap);
   return fail(EAS_ERR_UNSUPPORTED, "head_dim %d", hd);
