@@ -122,3 +122,32 @@ def test_attention_block_diagonal(hd, H, lens, impl):
     assert err <= 2e-2, err
     out2, _ = P.kernel_attention(_dev(qkv), cu, H, hd, impl=impl, sm_budget=3)
     assert torch.equal(out, out2)
+
+
+@pytest.mark.parametrize("H", [1, 2, 5, 16])
+def test_attention_dual_head_units(H):
+    """head_dim 64, items with an odd number of 128-row query tiles: their last tiles of two adjacent heads share a
+    unit (with an odd head count the last head's tile stays alone); items with an even count in the same launch keep
+    the ordinary units.  The tcgen05 kernel must agree with the oracle and, bit for bit, with itself at another budget;
+    the register-tile kernel (impl 1) has no such units and serves as a second opinion."""
+    import paper_2609_31551_b200 as P
+    hd, lens = 64, [577, 65, 640, 320, 577, 128, 1]
+    rng = np.random.Generator(np.random.PCG64(900 + H))
+    T, d = sum(lens), H * hd
+    qkv = _bf16_exact(rng, (T, 3 * d))
+    qkv[:, : 2 * d] *= 1.5
+    qkv = S.round_to_bf16(qkv)
+    cu = np.concatenate([[0], np.cumsum(lens)]).astype(np.int32)
+    q = O._t(qkv)
+    ref = torch.cat([O.attention_one_item(q[a:b, :d].reshape(-1, H, hd), q[a:b, d:2 * d].reshape(-1, H, hd),
+                                          q[a:b, 2 * d:].reshape(-1, H, hd)) for a, b in zip(cu[:-1], cu[1:])])
+    out, status = P.kernel_attention(_dev(qkv), cu, H, hd, impl=0)
+    torch.cuda.synchronize()
+    assert int(status[0]) == 0
+    err = (out.double().cpu() - ref).abs()
+    assert err.max() <= 2e-2, (err.max(), np.unravel_index(int(err.argmax()), err.shape))
+    for budget in (1, 7, 40):
+        out2, _ = P.kernel_attention(_dev(qkv), cu, H, hd, impl=0, sm_budget=budget)
+        assert torch.equal(out, out2), budget
+    out3, _ = P.kernel_attention(_dev(qkv), cu, H, hd, impl=1)
+    assert (out.float() - out3.float()).abs().max() <= 2e-2
