@@ -125,6 +125,14 @@ def test_degenerate_micro_batches():
     ref, _, _ = O.encode_microbatch(cfg, w, many)
     got, _ = G.run_gpu(enc, cfg, many)
     G.assert_parity(got, ref, "64 tiny images")
+    most = S.make_items(cfg, [(1, 28 * (1 + i % 2), 28 * (1 + i % 5)) for i in range(128)], seed=4)   # EAS_MAX_ITEMS
+    ref, _, _ = O.encode_microbatch(cfg, w, most)
+    got, _ = G.run_gpu(enc, cfg, most)
+    G.assert_parity(got, ref, "128 items, the most a call takes")
+    import paper_2609_31551_b200 as P
+    with pytest.raises(P.EasError) as e:
+        G.run_gpu(enc, cfg, S.make_items(cfg, [(1, 28, 28)] * 129, seed=5))
+    assert e.value.status == 1 and "n_items" in str(e.value)
     cfg4 = S.get_config("c4", n_layers=1)
     w4, enc4 = _make(cfg4)
     a = S.make_items(cfg4, [(2, 128, 1)] * 3, seed=3)             # 1 token per clip
