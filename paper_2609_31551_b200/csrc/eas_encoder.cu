@@ -558,22 +558,36 @@ static eas_status launch_gemm(const GemmCall& g, int budget, cudaStream_t stream
   const Linear& L = *g.lin;
   if (g.M <= 0) return EAS_OK;
   if (L.N % 32 != 0 || g.a_run % kBK != 0) return fail(EAS_ERR_UNSUPPORTED, "GEMM needs N %% 32 == 0 and K %% 64 == 0 (N=%d, K=%lld)", L.N, static_cast<long long>(g.a_run));
-  // CTA pairs (two SMs on one 256x256 tile, each loading half of the weight tile) whenever two SMs are available
-  const int ctas = budget >= 2 ? 2 : 1;
+  // Tile shape: one CTA per 128x256 tile, a CTA pair per 256x256 tile, or a pair per wide 256x512 tile.  All three
+  // accumulate every output element over K in the same order, so the results are bit-identical and this is a pure
+  // speed choice: estimated time = waves x time of one tile.  The per-k-block times are measured on B200 with each
+  // shape forced over the encoder's GEMM shapes (M = 1154 ... 24000): the main loop is bound by the L2 -> SM fabric,
+  // so a 64-wide k-block takes 0.46 us (single CTA), 0.43 us (pair) or 0.75 us for twice the columns (wide pair),
+  // whatever the SM clock; the wide tile's epilogue (about 4 us) does not overlap the next main loop.  What decides
+  // in practice is the wave count: at M = 4616 (c1, micro-batch 8) the out-projection is 2 half-empty waves of
+  // pair tiles but exactly 1 wave of single-CTA tiles.
   const bool tma_out = g.row_map == nullptr && g.pos == nullptr && (g.resid == nullptr || g.resid == g.out);
-  // wide 256x512 tiles for long reductions whose output splits evenly into 512-column blocks
   const int64_t k_total = g.a_run * g.taps;
-  bool wide = ctas == 2 && tma_out && g.act != ACT_SWIGLU && k_total >= 2048 && L.N % 512 == 0 &&
-              gemm_kernel_for(g.act, g.out_fp32, 3) != nullptr;
-  if (wide) {
-    // only when the half as many, twice as large tiles still fill the CTA pairs about as evenly (a wide tile is worth
-    // roughly 15 % per unit of work); the two tilings give bit-identical results, so this is a pure speed choice
+  const double kb = static_cast<double>(k_total / kBK);
+  auto waves = [](long long tiles, long long slots) { return static_cast<double>((tiles + slots - 1) / slots); };
+  const long long n256 = (L.N + kBN - 1) / kBN;
+  int ctas = 1;
+  bool wide = false;
+  if (budget >= 2) {
     const long long pairs = budget / 2;
-    const long long mg = (g.M + 2 * kBM - 1) / (2 * kBM);
-    const long long t_n = mg * ((L.N + kBN - 1) / kBN), t_w = mg * (L.N / (2 * kBN));
-    const double eff_n = static_cast<double>(t_n) / static_cast<double>(((t_n + pairs - 1) / pairs) * pairs);
-    const double eff_w = static_cast<double>(t_w) / static_cast<double>(((t_w + pairs - 1) / pairs) * pairs);
-    wide = t_w >= pairs && eff_w * 1.15 >= eff_n;
+    const long long m128 = (g.M + kBM - 1) / kBM, m256 = (g.M + 2 * kBM - 1) / (2 * kBM);
+    const double cost_single = waves(m128 * n256, budget) * kb * 0.46;
+    const double cost_pair = waves(m256 * n256, pairs) * kb * 0.43;
+    ctas = cost_single < cost_pair ? 1 : 2;
+    // wide tiles: long reductions whose output splits evenly into 512-column blocks, plain TMA-stored epilogue
+    if (tma_out && g.act != ACT_SWIGLU && k_total >= 2048 && L.N % 512 == 0 && gemm_kernel_for(g.act, g.out_fp32, 3) != nullptr) {
+      const double cost_wide = waves(m256 * (L.N / (2 * kBN)), pairs) * (kb * 0.75 + 4.0);
+      if (cost_wide < std::min(cost_single, cost_pair)) { ctas = 2; wide = true; }
+    }
+#ifdef EAS_GEMM_FORCE_TILE   // calibration builds only: 1 single CTA, 2 pair, 3 wide pair (where a wide kernel exists)
+    ctas = EAS_GEMM_FORCE_TILE == 1 ? 1 : 2;
+    wide = EAS_GEMM_FORCE_TILE == 3 && tma_out && g.act != ACT_SWIGLU && L.N % 512 == 0 && gemm_kernel_for(g.act, g.out_fp32, 3) != nullptr;
+#endif
   }
   const int tile_n = wide ? 2 * kBN : kBN;
   GemmParams p{};
