@@ -87,6 +87,22 @@ static eas_status make_a_tmap(CUtensorMap* m, const void* a, int64_t run, int64_
   return make_tmap(m, a, 3, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B);
 }
 
+// "Deep" maps: the same matrices seen as {64 columns, rows, K/64 blocks}, so that ONE box {64, rows, 2} brings two
+// 64-wide k-blocks, each landing as its own swizzle-atom block [rows x 128 bytes] (see GemmCfg).  A k-block index
+// past K/64 is filled with zeros.
+static eas_status make_w_tmap_deep(CUtensorMap* m, const void* w, int64_t N, int64_t K, uint32_t box_rows) {
+  const uint64_t dims[3] = {kBK, static_cast<uint64_t>(N), static_cast<uint64_t>(K / kBK)};
+  const uint64_t strides[2] = {static_cast<uint64_t>(K) * 2, kBK * 2};
+  const uint32_t box[3] = {kBK, box_rows, 2};
+  return make_tmap(m, w, 3, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B);
+}
+static eas_status make_a_tmap_deep(CUtensorMap* m, const void* a, int64_t run, int64_t row_elems, int64_t rows) {
+  const uint64_t dims[3] = {kBK, static_cast<uint64_t>(rows), static_cast<uint64_t>(run / kBK)};
+  const uint64_t strides[2] = {static_cast<uint64_t>(row_elems) * 2, kBK * 2};
+  const uint32_t box[3] = {kBK, kBM, 2};
+  return make_tmap(m, a, 3, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B);
+}
+
 // output [rows, ld] as a store / reduce target: 32-row boxes whose rows are 128 bytes (64 bf16 or 32 fp32)
 static eas_status make_out_tmap(CUtensorMap* m, const void* out, bool fp32, int64_t cols, int64_t ld, int64_t rows) {
   PFN_cuTensorMapEncodeTiled_v12000 fn = get_encode_fn();
@@ -109,6 +125,7 @@ struct Linear {
   int N = 0, K = 0;
   CUtensorMap tmap;        // box of 256 weight rows
   CUtensorMap tmap_half;   // box of 128 weight rows (CTA-pair kernel)
+  CUtensorMap tmap_deep, tmap_half_deep;   // the same for the deep kernels (two k-blocks per box)
 };
 struct Layer {
   const bf16 *n1g = nullptr, *n1b = nullptr, *n2g = nullptr, *n2b = nullptr;
@@ -259,16 +276,25 @@ static eas_status relayout(bf16* dst, const bf16* src, const bf16* src2, long lo
 
 static eas_status finish_linear(Linear& L) {
   EAS_TRY(make_w_tmap(&L.tmap, L.w, L.N, L.K, kBN));
-  return make_w_tmap(&L.tmap_half, L.w, L.N, L.K, kBN / 2);
+  EAS_TRY(make_w_tmap(&L.tmap_half, L.w, L.N, L.K, kBN / 2));
+  EAS_TRY(make_w_tmap_deep(&L.tmap_deep, L.w, L.N, L.K, kBN));
+  return make_w_tmap_deep(&L.tmap_half_deep, L.w, L.N, L.K, kBN / 2);
 }
 
 typedef void (*GemmKernel)(GemmParams);
-// ctas: 1 = one CTA per 128x256 tile; 2 = CTA pair per 256x256 tile; 3 = CTA pair per 256x512 tile ("wide")
-static GemmKernel gemm_kernel_for(int act, int out_fp32, int ctas) {
+// ctas: 1 = one CTA per 128x256 tile; 2 = CTA pair per 256x256 tile; 3 = CTA pair per 256x512 tile ("wide");
+// deep (pair tiles only): two 64-wide k-blocks per stage and TMA operation
+static GemmKernel gemm_kernel_for(int act, int out_fp32, int ctas, bool deep = false) {
   if (ctas == 3) {
     if (act == ACT_NONE && !out_fp32) return gemm_kernel<ACT_NONE, OUT_BF16, 2, 2>;
     if (act == ACT_GELU && !out_fp32) return gemm_kernel<ACT_GELU, OUT_BF16, 2, 2>;
     if (act == ACT_NONE && out_fp32) return gemm_kernel<ACT_NONE, OUT_F32, 2, 2>;
+  } else if (ctas == 2 && deep) {
+    if (act == ACT_NONE && !out_fp32) return gemm_kernel<ACT_NONE, OUT_BF16, 2, 1, 2>;
+    if (act == ACT_GELU && !out_fp32) return gemm_kernel<ACT_GELU, OUT_BF16, 2, 1, 2>;
+    if (act == ACT_SWIGLU && !out_fp32) return gemm_kernel<ACT_SWIGLU, OUT_BF16, 2, 1, 2>;
+    if (act == ACT_NONE && out_fp32) return gemm_kernel<ACT_NONE, OUT_F32, 2, 1, 2>;
+    if (act == ACT_GELU && out_fp32) return gemm_kernel<ACT_GELU, OUT_F32, 2, 1, 2>;
   } else if (ctas == 2) {
     if (act == ACT_NONE && !out_fp32) return gemm_kernel<ACT_NONE, OUT_BF16, 2, 1>;
     if (act == ACT_GELU && !out_fp32) return gemm_kernel<ACT_GELU, OUT_BF16, 2, 1>;
@@ -285,13 +311,14 @@ static GemmKernel gemm_kernel_for(int act, int out_fp32, int ctas) {
   return nullptr;
 }
 static eas_status set_kernel_attributes() {
-  for (int ctas = 1; ctas <= 3; ++ctas)
-    for (int act = 0; act < 3; ++act)
-      for (int f32 = 0; f32 < 2; ++f32) {
-        GemmKernel k = gemm_kernel_for(act, f32, ctas);
-        if (k != nullptr)
-          CUDA_TRY(cudaFuncSetAttribute(reinterpret_cast<const void*>(k), cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmemBytes));
-      }
+  for (int deep = 0; deep < 2; ++deep)
+    for (int ctas = 1; ctas <= 3; ++ctas)
+      for (int act = 0; act < 3; ++act)
+        for (int f32 = 0; f32 < 2; ++f32) {
+          GemmKernel k = gemm_kernel_for(act, f32, ctas, deep != 0);
+          if (k != nullptr)
+            CUDA_TRY(cudaFuncSetAttribute(reinterpret_cast<const void*>(k), cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmemBytes));
+        }
   return EAS_OK;
 }
 
@@ -561,10 +588,10 @@ static eas_status launch_gemm(const GemmCall& g, int budget, cudaStream_t stream
   // Tile shape: one CTA per 128x256 tile, a CTA pair per 256x256 tile, or a pair per wide 256x512 tile.  All three
   // accumulate every output element over K in the same order, so the results are bit-identical and this is a pure
   // speed choice: estimated time = waves x time of one tile.  The per-k-block times are measured on B200 with each
-  // shape forced over the encoder's GEMM shapes (M = 1154 ... 24000): the main loop is bound by the L2 -> SM fabric,
-  // so a 64-wide k-block takes 0.46 us (single CTA), 0.43 us (pair) or 0.75 us for twice the columns (wide pair),
-  // whatever the SM clock; the wide tile's epilogue (about 4 us) does not overlap the next main loop.  What decides
-  // in practice is the wave count: at M = 4616 (c1, micro-batch 8) the out-projection is 2 half-empty waves of
+  // shape forced over the encoder's GEMM shapes (M = 1154 ... 24000): a 64-wide k-block takes 0.47 us (single CTA),
+  // 0.40 us (pair, deep stages; 0.43 for the convolutions' shallow ones) or 0.75 us for twice the columns (wide
+  // pair); the wide tile's epilogue (about 4 us) does not overlap the next main loop.  What decides in practice is
+  // the wave count: at M = 4616 (c1, micro-batch 8) the out-projection is 2 half-empty waves of
   // pair tiles but exactly 1 wave of single-CTA tiles.
   const bool tma_out = g.row_map == nullptr && g.pos == nullptr && (g.resid == nullptr || g.resid == g.out);
   const int64_t k_total = g.a_run * g.taps;
@@ -576,8 +603,8 @@ static eas_status launch_gemm(const GemmCall& g, int budget, cudaStream_t stream
   if (budget >= 2) {
     const long long pairs = budget / 2;
     const long long m128 = (g.M + kBM - 1) / kBM, m256 = (g.M + 2 * kBM - 1) / (2 * kBM);
-    const double cost_single = waves(m128 * n256, budget) * kb * 0.46;
-    const double cost_pair = waves(m256 * n256, pairs) * kb * 0.43;
+    const double cost_single = waves(m128 * n256, budget) * kb * 0.47;
+    const double cost_pair = waves(m256 * n256, pairs) * kb * (g.conv_stride == 1 && g.taps == 1 ? 0.40 : 0.43);
     ctas = cost_single < cost_pair ? 1 : 2;
     // wide tiles: long reductions whose output splits evenly into 512-column blocks, plain TMA-stored epilogue
     if (tma_out && g.act != ACT_SWIGLU && k_total >= 2048 && L.N % 512 == 0 && gemm_kernel_for(g.act, g.out_fp32, 3) != nullptr) {
@@ -590,12 +617,17 @@ static eas_status launch_gemm(const GemmCall& g, int budget, cudaStream_t stream
 #endif
   }
   const int tile_n = wide ? 2 * kBN : kBN;
+  // pair tiles of plain GEMMs run the deep kernel (two k-blocks per stage and TMA operation: 8 % faster at K = 1024);
+  // single-CTA and wide tiles would be left with two 96 KB stages and measured no better, and convolutions walk their
+  // taps as 64-wide k-blocks
+  const bool deep = g.conv_stride == 1 && g.taps == 1 && ctas == 2 && !wide;
   GemmParams p{};
-  EAS_TRY(make_a_tmap(&p.tma_a, g.A, g.a_run, g.a_row_elems, g.conv_stride, g.a_rows));
-  p.tma_b = ctas == 2 ? L.tmap_half : L.tmap;
+  if (deep) EAS_TRY(make_a_tmap_deep(&p.tma_a, g.A, g.a_run, g.a_row_elems, g.a_rows));
+  else EAS_TRY(make_a_tmap(&p.tma_a, g.A, g.a_run, g.a_row_elems, g.conv_stride, g.a_rows));
+  p.tma_b = deep ? (ctas == 2 ? L.tmap_half_deep : L.tmap_deep) : (ctas == 2 ? L.tmap_half : L.tmap);
   p.M = g.M; p.N = L.N;
   p.kb_per_tap = static_cast<int>(g.a_run / kBK);
-  p.k_blocks = p.kb_per_tap * g.taps;
+  p.k_blocks = deep ? (p.kb_per_tap + 1) / 2 : p.kb_per_tap * g.taps;
   p.conv_stride = g.conv_stride;
   p.m_blocks = (g.M + kBM * ctas - 1) / (kBM * ctas);
   p.n_blocks = (L.N + tile_n - 1) / tile_n;
@@ -611,7 +643,7 @@ static eas_status launch_gemm(const GemmCall& g, int budget, cudaStream_t stream
     EAS_TRY(make_out_tmap(&p.tma_out, g.out, g.out_fp32 != 0, out_cols, g.ldo, g.M));
   }
   const int tiles = p.m_blocks * p.n_blocks;
-  GemmKernel kern = gemm_kernel_for(g.act, g.out_fp32, wide ? 3 : ctas);
+  GemmKernel kern = gemm_kernel_for(g.act, g.out_fp32, wide ? 3 : ctas, deep);
   if (kern == nullptr) return fail(EAS_ERR_UNSUPPORTED, "no GEMM epilogue for act=%d out_fp32=%d", g.act, g.out_fp32);
   return launch_kernel(kern, std::min(budget / ctas, tiles) * ctas, kGemmThreads, kGemmSmemBytes, stream, p, ctas);
 }

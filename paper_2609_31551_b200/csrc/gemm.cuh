@@ -23,10 +23,15 @@ constexpr int kABytes = kBM * kBK * 2;            // 16 KB: 128 rows of A
 // NW = 2 ("wide", CTA pairs only): the pair owns a 256x512 tile, i.e. two 256-column accumulators fed by the same
 // A tile.  That cuts the operand bytes per FLOP by a quarter (the L2 -> SM path is what bounds the main loop) at the
 // price of a single accumulator set: the epilogue no longer overlaps the next main loop, so it pays for large K only.
-template <int CTAS, int NW> struct GemmCfg {
-  static constexpr int kBBytes = (kBN / CTAS) * kBK * 2 * NW;
-  static constexpr int kStageBytes = kABytes + kBBytes;
-  static constexpr int kStages = CTAS == 2 ? (NW == 2 ? 4 : 6) : 4;
+// KD = 2 ("deep"): a stage holds TWO 64-wide k-blocks of each operand, fetched by ONE TMA operation per operand
+// (a 3-D box {64 columns, rows, 2 k-blocks}, which lands as two consecutive swizzle-atom blocks).  Measured on B200:
+// what a CTA can pull from L2 is set by the number of TMA operations in flight, not by their bytes (two 16 KB
+// boxes per 0.46 us, but also two 32 KB boxes per 0.47 us), so deep stages double the operand rate and move the main
+// loop from the load path to the tensor pipe.  Half as many, twice as large stages: same shared memory.
+template <int CTAS, int NW, int KD = 1> struct GemmCfg {
+  static constexpr int kBBytes = (kBN / CTAS) * kBK * 2 * NW;      // per 64-wide k-block
+  static constexpr int kStageBytes = (kABytes + kBBytes) * KD;
+  static constexpr int kStages = (CTAS == 2 ? (NW == 2 ? 4 : 6) : 4) / KD;
   static constexpr int kAccBuffers = NW == 2 ? 1 : 2;
 };
 constexpr int kMaxStages = 6;
@@ -42,12 +47,12 @@ enum { ACT_NONE = 0, ACT_GELU = 1, ACT_SWIGLU = 2 };
 enum { OUT_BF16 = 0, OUT_F32 = 1 };
 
 struct alignas(64) GemmParams {
-  CUtensorMap tma_a;      // 3-D: {K-run, phase, rows}; box {64, 1, 128}
-  CUtensorMap tma_b;      // 2-D: {K, N}; box {64, 256} (one CTA per tile) or {64, 128} (CTA pair)
+  CUtensorMap tma_a;      // 3-D: {K-run, phase, rows}; box {64, 1, 128}.  Deep kernels: {64, rows, K/64}; box {64, 128, 2}
+  CUtensorMap tma_b;      // 2-D: {K, N}; box {64, 256} (one CTA per tile) or {64, 128} (CTA pair).  Deep: {64, N, K/64}; box {64, rows, 2}
   CUtensorMap tma_out;    // 2-D over out: box {64 bf16 | 32 fp32, 32 rows}, 128-byte swizzle (valid if use_tma_out)
   int use_tma_out;        // 1: epilogue stages 32-row sub-tiles in shared memory and stores them with TMA
   int M, N;               // rows of A walked by tiles; rows of W
-  int k_blocks;           // K / 64 (K padded with zeros by the caller or by TMA fill)
+  int k_blocks;           // k-steps: K / 64, or ceil(K / 128) for the deep kernels (TMA fills past K with zeros)
   int kb_per_tap;         // k-blocks per convolution tap (== k_blocks for a plain GEMM)
   int conv_stride;        // 1 for a plain GEMM; row stride of a convolution otherwise
   int m_blocks, n_blocks; // m_blocks counts 128-row blocks (one CTA per tile) or 256-row blocks (CTA pair)
@@ -74,12 +79,15 @@ __device__ __forceinline__ void tile_coords(int tile, int m_blocks, int n_blocks
   mb = panel * kPanelM + (within - nb * rows_here);
 }
 
-template <int ACT, int OUT, int CTAS, int NW>
+template <int ACT, int OUT, int CTAS, int NW, int KD = 1>
 __global__ void __launch_bounds__(kGemmThreads, 1) gemm_kernel(const __grid_constant__ GemmParams p) {
   static_assert(NW == 1 || (CTAS == 2 && ACT != ACT_SWIGLU), "wide tiles: CTA pairs, no gated epilogue");
-  constexpr int kStages = GemmCfg<CTAS, NW>::kStages;
-  constexpr int kStageBytes = GemmCfg<CTAS, NW>::kStageBytes;
-  constexpr int kAccBuffers = GemmCfg<CTAS, NW>::kAccBuffers;
+  static_assert(KD == 1 || KD == 2, "one or two 64-wide k-blocks per stage");
+  constexpr int kStages = GemmCfg<CTAS, NW, KD>::kStages;
+  constexpr int kStageBytes = GemmCfg<CTAS, NW, KD>::kStageBytes;
+  constexpr int kAccBuffers = GemmCfg<CTAS, NW, KD>::kAccBuffers;
+  constexpr int kBRows = kBN / CTAS;               // weight rows per CTA and 256-column accumulator
+  constexpr int kBAtom = kBRows * kBK * 2;         // bytes of one 64-wide k-block of those rows
   constexpr int kTileN = kBN * NW;                 // output columns of a tile
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   // 1024-byte alignment: the 128-byte swizzle pattern repeats every 8 rows of 128 bytes
@@ -135,7 +143,22 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_kernel(const __grid_cons
           const uint32_t ph = (it / kStages) & 1u;
           if (!mbar_wait(&empty_bar[s], ph ^ 1u, abort_flag)) { ok = false; break; }
           uint8_t* sa = smem + s * kStageBytes;
-          uint8_t* sb = sa + kABytes;
+          uint8_t* sb = sa + kABytes * KD;
+          if (KD == 2) {
+            // deep stage (plain GEMM only): [A k-block 0][A k-block 1][B ...] from one 3-D box per operand
+            if (CTAS == 2) {
+              if (cta_rank == 0) mbar_expect_tx(&full_bar[s], 2 * kStageBytes);
+              tma_load_3d_pair(sa, &p.tma_a, &full_bar[s], 0, mb * kBM, kb * KD);
+#pragma unroll
+              for (int h = 0; h < NW; ++h)
+                tma_load_3d_pair(sb + h * kBAtom * KD, &p.tma_b, &full_bar[s], 0, nb * kTileN + h * kBN + cta_rank * kBRows, kb * KD);
+            } else {
+              mbar_expect_tx(&full_bar[s], kStageBytes);
+              tma_load_3d(sa, &p.tma_a, &full_bar[s], 0, mb * kBM, kb * KD);
+              tma_load_3d(sb, &p.tma_b, &full_bar[s], 0, nb * kBN, kb * KD);
+            }
+            continue;
+          }
           const int tap = kb / p.kb_per_tap;
           const int kx = (kb - tap * p.kb_per_tap) * kBK;
           if (CTAS == 2) {
@@ -179,19 +202,22 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_kernel(const __grid_cons
           if (!mbar_wait(&full_bar[s], ph, abort_flag)) { ok = false; break; }
           tc_fence_after_sync();
           const uint32_t a_addr = smem_u32(smem + s * kStageBytes);
-          const uint32_t b_addr = a_addr + kABytes;
-          const uint64_t adesc = make_smem_desc(a_addr, 16, 1024, kSwizzle128B);
-          const uint64_t bdesc = make_smem_desc(b_addr, 16, 1024, kSwizzle128B);
+          const uint32_t b_addr = a_addr + kABytes * KD;
 #pragma unroll
-          for (int k = 0; k < kBK / 16; ++k) {
-            // advancing 16 bf16 = 32 bytes along K inside the swizzle atom: +2 in the (>>4) address field
-            if (CTAS == 2) {
+          for (int a = 0; a < KD; ++a) {         // the 64-wide k-blocks of the stage: one swizzle-atom block each
+            const uint64_t adesc = make_smem_desc(a_addr + a * kABytes, 16, 1024, kSwizzle128B);
+            const uint64_t bdesc = make_smem_desc(b_addr + a * kBAtom, 16, 1024, kSwizzle128B);
 #pragma unroll
-              for (int h = 0; h < NW; ++h)   // second accumulator: the next 128 weight rows of each CTA, 16 KB further
-                umma_bf16_ss_pair(tmem_d + h * kBN, adesc + 2 * k, bdesc + 2 * k + h * ((kBN / 2) * kBK * 2 / 16), idesc,
-                                  (kb | k) != 0);
-            } else {
-              umma_bf16_ss(tmem_d, adesc + 2 * k, bdesc + 2 * k, idesc, (kb | k) != 0);
+            for (int k = 0; k < kBK / 16; ++k) {
+              // advancing 16 bf16 = 32 bytes along K inside the swizzle atom: +2 in the (>>4) address field
+              if (CTAS == 2) {
+#pragma unroll
+                for (int h = 0; h < NW; ++h)   // second accumulator: the next 128 weight rows of each CTA
+                  umma_bf16_ss_pair(tmem_d + h * kBN, adesc + 2 * k, bdesc + 2 * k + h * (kBAtom * KD / 16), idesc,
+                                    (kb | a | k) != 0);
+              } else {
+                umma_bf16_ss(tmem_d, adesc + 2 * k, bdesc + 2 * k, idesc, (kb | a | k) != 0);
+              }
             }
           }
           // frees the stage (in both CTAs of a pair) once these UMMAs have read it
