@@ -1,6 +1,6 @@
 // Persistent bf16 GEMM for sm_100a:  D[M,N] = A[M,K] * W[N,K]^T  with a fused epilogue.
 //
-//   warp 0      TMA producer: 128x64 A tiles and 256x64 W tiles into a 4-stage shared-memory ring
+//   warp 0, 10  TMA producers (A tiles, W tiles): 128x64 A tiles and 256x64 W tiles into a shared-memory ring
 //   warp 1      UMMA issuer: tcgen05.mma 128x256x16, fp32 accumulators in TMEM, two accumulator
 //               buffers (2 x 256 columns) so that the epilogue of tile i overlaps the main loop of tile i+1
 //   warps 2..9  epilogue: tcgen05.ld -> bias / activation / rotary -> swizzled shared-memory staging -> TMA store
@@ -16,7 +16,8 @@ namespace eas {
 
 constexpr int kBM = 128, kBN = 256, kBK = 64;
 constexpr int kEpiWarps = 8;
-constexpr int kGemmThreads = 64 + 32 * kEpiWarps;
+constexpr int kGemmThreads = 64 + 32 * kEpiWarps + 32;   // + the second producer warp
+constexpr int kProducerBWarp = 2 + kEpiWarps;
 constexpr int kABytes = kBM * kBK * 2;            // 16 KB: 128 rows of A
 // one CTA per tile: a stage holds A (16 KB) + the whole 256-row weight tile (32 KB), 4 stages;
 // CTA pair per 256x256 tile: a stage holds A (16 KB) + this CTA's 128 weight rows (16 KB), 6 stages
@@ -129,8 +130,12 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_kernel(const __grid_cons
   pdl_launch_dependents();   // the next kernel may set itself up while this one runs
   pdl_wait();                // everything before this kernel in the stream is complete and visible
 
-  if (warp == 0) {
-    // ------------------------------------------------------------------ producer
+  if (warp == 0 || warp == kProducerBWarp) {
+    // ------------------------------------------------------------------ producers: warp 0 loads A, the last warp B
+    // Issuing a TMA operation occupies the issuing thread for some 70 ns, and that is what bounds the operand rate
+    // of a CTA (measured: a step of two 32 KB boxes takes 476 ns from one thread, 396 ns from two), so the two
+    // operands have a thread each.  The A thread announces the bytes of the whole stage.
+    const bool do_a = warp == 0, do_b = warp != 0;
     if (lane == 0) {
       uint32_t it = 0;
       bool ok = true;
@@ -144,35 +149,35 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_kernel(const __grid_cons
           if (!mbar_wait(&empty_bar[s], ph ^ 1u, abort_flag)) { ok = false; break; }
           uint8_t* sa = smem + s * kStageBytes;
           uint8_t* sb = sa + kABytes * KD;
+          // both CTAs' loads of a pair complete on the leader's barrier; the leader announces the bytes of both
+          if (do_a && cta_rank == 0) mbar_expect_tx(&full_bar[s], CTAS * kStageBytes);
           if (KD == 2) {
             // deep stage (plain GEMM only): [A k-block 0][A k-block 1][B ...] from one 3-D box per operand
             if (CTAS == 2) {
-              if (cta_rank == 0) mbar_expect_tx(&full_bar[s], 2 * kStageBytes);
-              tma_load_3d_pair(sa, &p.tma_a, &full_bar[s], 0, mb * kBM, kb * KD);
+              if (do_a) tma_load_3d_pair(sa, &p.tma_a, &full_bar[s], 0, mb * kBM, kb * KD);
+              if (do_b) {
 #pragma unroll
-              for (int h = 0; h < NW; ++h)
-                tma_load_3d_pair(sb + h * kBAtom * KD, &p.tma_b, &full_bar[s], 0, nb * kTileN + h * kBN + cta_rank * kBRows, kb * KD);
+                for (int h = 0; h < NW; ++h)
+                  tma_load_3d_pair(sb + h * kBAtom * KD, &p.tma_b, &full_bar[s], 0, nb * kTileN + h * kBN + cta_rank * kBRows, kb * KD);
+              }
             } else {
-              mbar_expect_tx(&full_bar[s], kStageBytes);
-              tma_load_3d(sa, &p.tma_a, &full_bar[s], 0, mb * kBM, kb * KD);
-              tma_load_3d(sb, &p.tma_b, &full_bar[s], 0, nb * kBN, kb * KD);
+              if (do_a) tma_load_3d(sa, &p.tma_a, &full_bar[s], 0, mb * kBM, kb * KD);
+              if (do_b) tma_load_3d(sb, &p.tma_b, &full_bar[s], 0, nb * kBN, kb * KD);
             }
             continue;
           }
           const int tap = kb / p.kb_per_tap;
           const int kx = (kb - tap * p.kb_per_tap) * kBK;
           if (CTAS == 2) {
-            // both CTAs' loads complete on the leader's barrier; the leader announces the bytes of both
-            if (cta_rank == 0) mbar_expect_tx(&full_bar[s], 2 * kStageBytes);
-            tma_load_3d_pair(sa, &p.tma_a, &full_bar[s], kx, tap % p.conv_stride, mb * kBM + tap / p.conv_stride);
+            if (do_a) tma_load_3d_pair(sa, &p.tma_a, &full_bar[s], kx, tap % p.conv_stride, mb * kBM + tap / p.conv_stride);
+            if (do_b) {
 #pragma unroll
-            for (int h = 0; h < NW; ++h)
-              tma_load_2d_pair(sb + h * (kBN / 2) * kBK * 2, &p.tma_b, &full_bar[s], kb * kBK,
-                               nb * kTileN + h * kBN + cta_rank * (kBN / 2));
+              for (int h = 0; h < NW; ++h)
+                tma_load_2d_pair(sb + h * kBAtom, &p.tma_b, &full_bar[s], kb * kBK, nb * kTileN + h * kBN + cta_rank * kBRows);
+            }
           } else {
-            mbar_expect_tx(&full_bar[s], kStageBytes);
-            tma_load_3d(sa, &p.tma_a, &full_bar[s], kx, tap % p.conv_stride, mb * kBM + tap / p.conv_stride);
-            tma_load_2d(sb, &p.tma_b, &full_bar[s], kb * kBK, nb * kBN);
+            if (do_a) tma_load_3d(sa, &p.tma_a, &full_bar[s], kx, tap % p.conv_stride, mb * kBM + tap / p.conv_stride);
+            if (do_b) tma_load_2d(sb, &p.tma_b, &full_bar[s], kb * kBK, nb * kBN);
           }
         }
       }
@@ -228,7 +233,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_kernel(const __grid_cons
         }
       }
     }
-  } else {
+  } else if (warp < kProducerBWarp) {
     // ------------------------------------------------------------------ epilogue
     const int ew = warp - 2;                    // 0..7
     const int quarter = warp & 3;               // TMEM lane quarter this warp may read
