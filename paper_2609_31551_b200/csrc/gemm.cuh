@@ -320,6 +320,33 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_kernel(const __grid_cons
           }
         };
 
+        if (OUT == OUT_F32) {
+          // fp32 output: 32 columns = one 128-byte staging row, so every 32-column chunk is a sub-tile (and a TMA
+          // operation) of its own.  One chunk per round, the next chunk's TMEM load in flight meanwhile, so that the
+          // wait for the previous operation to release the staging buffer falls behind a load and the chunk's math.
+          constexpr int kChunks = 4 * NW;
+          uint32_t r[32];
+          __syncwarp();
+          tmem_ld_32x32(taddr, r);
+#pragma unroll 1
+          for (int c = 0; c < kChunks; ++c) {
+            tmem_ld_wait();
+            float v[32];
+#pragma unroll
+            for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+            if (c + 1 < kChunks) {
+              __syncwarp();
+              tmem_ld_32x32(taddr + (c + 1) * 32, r);
+            }
+            finish_chunk(v, c);
+            const int col0 = nb * kTileN + half * (128 * NW) + c * 32;
+            staging_free();
+#pragma unroll
+            for (int q = 0; q < 8; ++q)
+              *reinterpret_cast<float4*>(srow + ((q ^ sw) << 4)) = make_float4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
+            if (col0 < p.N) store_subtile(col0);
+          }
+        } else {
 #pragma unroll 1
         for (int pr = 0; pr < 2 * NW; ++pr) {       // two chunks (64 accumulator columns) per round
           uint32_t r0[32], r1[32];
@@ -373,6 +400,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_kernel(const __grid_cons
             }
             if (col0 < p.N) store_subtile(col0);
           }
+        }
         }
         release_accumulator(acc);
         continue;
