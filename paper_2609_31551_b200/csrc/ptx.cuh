@@ -278,26 +278,24 @@ __device__ __forceinline__ uint64_t fmul2(uint64_t a, uint64_t b) {
   asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
   return d;
 }
-// GELU (erf form, same rational-exponential erf as gelu_erf) on two values at once with packed fp32x2 arithmetic
+// GELU (erf form, same rational-exponential erf as gelu_erf) on two values at once with packed fp32x2 arithmetic.
+// With z = |x| / sqrt(2), t = 1 / (1 + p z) and q = 0.5 poly(t) exp(-z^2) (so that erf(z) = 1 - 2 q):
+//   x >= 0:  gelu = 0.5 x (1 + erf z) = x - x q        x < 0:  gelu = 0.5 x (1 - erf z) = x q
+// i.e. gelu(x) = max(x, 0) - |x| q for both signs: no copysign, and the constants of z fold into the coefficients.
 __device__ __forceinline__ void gelu_erf_pair(float& x0, float& x1) {
-  const uint64_t x2 = pack2(x0, x1);
-  const uint64_t az2 = pack2(fabsf(x0) * 0.70710678118654752f, fabsf(x1) * 0.70710678118654752f);
+  const uint64_t nax2 = pack2(-fabsf(x0), -fabsf(x1));                                   // -|x|
   float d0, d1;
-  unpack2(ffma2(pack2(0.3275911f, 0.3275911f), az2, pack2(1.0f, 1.0f)), d0, d1);
+  unpack2(ffma2(pack2(-0.2316418882f, -0.2316418882f), nax2, pack2(1.0f, 1.0f)), d0, d1);   // 1 + 0.3275911 |x| / sqrt 2
   const uint64_t t2 = pack2(fast_rcp(d0), fast_rcp(d1));
-  uint64_t p2 = ffma2(pack2(1.061405429f, 1.061405429f), t2, pack2(-1.453152027f, -1.453152027f));
-  p2 = ffma2(p2, t2, pack2(1.421413741f, 1.421413741f));
-  p2 = ffma2(p2, t2, pack2(-0.284496736f, -0.284496736f));
-  p2 = ffma2(p2, t2, pack2(0.254829592f, 0.254829592f));
+  uint64_t p2 = ffma2(pack2(0.5307027145f, 0.5307027145f), t2, pack2(-0.7265760135f, -0.7265760135f));   // halved A&S 7.1.26
+  p2 = ffma2(p2, t2, pack2(0.7107068705f, 0.7107068705f));
+  p2 = ffma2(p2, t2, pack2(-0.142248368f, -0.142248368f));
+  p2 = ffma2(p2, t2, pack2(0.127414796f, 0.127414796f));
   p2 = fmul2(p2, t2);
   float e0, e1;
-  unpack2(fmul2(fmul2(az2, az2), pack2(-1.4426950408889634f, -1.4426950408889634f)), e0, e1);
-  const uint64_t e2 = pack2(fast_ex2(e0), fast_ex2(e1));
-  float r0, r1;
-  unpack2(ffma2(fmul2(p2, pack2(-1.0f, -1.0f)), e2, pack2(1.0f, 1.0f)), r0, r1);   // erf(|z|) = 1 - p e
-  const uint64_t erf2 = pack2(copysignf(r0, x0), copysignf(r1, x1));
-  const uint64_t hx2 = fmul2(x2, pack2(0.5f, 0.5f));
-  unpack2(ffma2(hx2, erf2, hx2), x0, x1);
+  unpack2(fmul2(fmul2(nax2, nax2), pack2(-0.7213475204f, -0.7213475204f)), e0, e1);      // -x^2 / 2 * log2(e)
+  const uint64_t q2 = fmul2(p2, pack2(fast_ex2(e0), fast_ex2(e1)));
+  unpack2(ffma2(nax2, q2, pack2(fmaxf(x0, 0.0f), fmaxf(x1, 0.0f))), x0, x1);             // max(x, 0) + (-|x|) q
 }
 __device__ __forceinline__ float silu_f(float x) {
   return x * fast_rcp(1.0f + fast_ex2(-1.4426950408889634f * x));
