@@ -8,7 +8,8 @@
 // (dual-head unit: A on head h, B on head h + 1, each with its own K/V tiles).
 //
 //   warp 0       TMA producer: Q tiles (double buffered across units), K/V tiles through a ring
-//   warp 1       UMMA issuer:  S = Q K^T (128x128x{64|80}) into TMEM, O += P V (128x{64|80}x128) in TMEM
+//   warp 1       UMMA issuer:  S = Q K^T (128 x keys x {64|80}) into TMEM, O += P V (128 x {64|80} x keys) in TMEM;
+//                keys per K/V tile: 128 for head_dim 64, 112 for head_dim 80 (see AttnTcSmem)
 //   warps 2, 3   idle (they complete the first warpgroup, whose registers are handed to the softmax warps)
 //   warps 4..7   softmax warpgroup of tile A: one thread per query row
 //   warps 8..11  softmax warpgroup of tile B
@@ -30,6 +31,8 @@ constexpr float kRescaleThreshold = 8.0f;
 struct AttnTcParams {
   CUtensorMap map_lo;   // qkv [T, 3d], box {64 columns, 128 rows}, 128-byte swizzle
   CUtensorMap map_hi;   // box {16 columns, 128 rows}, 32-byte swizzle (head_dim 80: columns 64..79)
+  CUtensorMap map_klo;  // qkv, box {64 columns, keys per K/V tile}, 128-byte swizzle (K and V tiles)
+  CUtensorMap map_khi;  // box {16 columns, keys per K/V tile}, 32-byte swizzle
   CUtensorMap map_out;  // out [T, d], box {64 columns, 32 rows}, 128-byte swizzle (store of a warp's 32 output rows)
   bf16* out;
   long long ldo;
@@ -44,21 +47,36 @@ struct AttnTcParams {
 
 // PT: the probabilities P live in tensor memory (the A operand of P V is read from there); otherwise they are
 // staged in shared memory.  With PT the 64 KB of P staging become extra K/V stages.
+#ifndef EAS_ATTN_KEYS_HD80
+#define EAS_ATTN_KEYS_HD80 112     // keys per K/V tile for head_dim 80 with P in tensor memory (128: the former layout)
+#endif
 template <int HD, bool PT>
 struct AttnTcSmem {
   static constexpr int HI = HD - 64;                       // 0 or 16 extra columns
-  static constexpr int kLoBytes = kTcTile * 128;           // 128 rows x 64 bf16
+  // Keys per K/V tile.  head_dim 80 with P in tensor memory takes 112: then S (2 x 112 columns), O (2 x 80) and
+  // dedicated P columns (2 x 56) fit the 512 columns of tensor memory together (496), P no longer has to re-use S's
+  // columns, and the next scores can be computed while P V of the current tile is still running, as for head_dim 64.
+  // With 128 keys the three would need 544 columns.
+  static constexpr int kKeys = (PT && HD != 64) ? EAS_ATTN_KEYS_HD80 : kTcTile;
+  static constexpr bool kNarrowO = PT && HD != 64 && kKeys < kTcTile;   // O is HD columns wide, P has its own columns
+  static constexpr int kLoBytes = kTcTile * 128;           // Q tile: 128 rows x 64 bf16
   static constexpr int kHiBytes = kTcTile * HI * 2;        // 128 rows x 16 bf16
-  static constexpr int kTileBytes = kLoBytes + kHiBytes;   // one Q, K or V tile
+  static constexpr int kTileBytes = kLoBytes + kHiBytes;   // one Q tile
+  static constexpr int kKLoBytes = kKeys * 128;            // K or V tile: keys x 64 bf16
+  static constexpr int kKHiBytes = kKeys * HI * 2;         // keys x 16 bf16
+  static constexpr int kKHiPad = (kKHiBytes + 1023) / 1024 * 1024;   // the next tile starts on a swizzle-atom boundary
+  static constexpr int kKTileBytes = kKLoBytes + kKHiPad;  // shared memory of one K tile
+  static constexpr int kKTxBytes = kKLoBytes + kKHiBytes;  // bytes its loads deliver
   static constexpr bool kStagedOut = PT && HD == 64;       // output rows leave through shared memory and TMA stores
   // With P in tensor memory and head_dim 80, V is loaded 128 columns wide (two 64-column boxes; the extra 48 columns
-  // belong to the next head, or are zero past the last one) so that P V is ONE N = 128 UMMA per 16 keys instead of an
-  // N = 64 plus an N = 16 one: the issuer is the bottleneck there and every UMMA costs about the same.  The surplus
-  // output columns 80..127 of O are never read.
+  // belong to the next head, or are zero past the last one) so that P V is ONE UMMA per 16 keys (N = 80 across the
+  // two swizzle atoms; N = 128 with 128-key tiles, whose surplus output columns are never read) instead of an N = 64
+  // plus an N = 16 one: the issuer is the bottleneck there and every UMMA costs about the same.
   static constexpr bool kWideV = PT && HD != 64;
-  static constexpr int kVBytes = kWideV ? 2 * kLoBytes : kTileBytes;
-  static constexpr int kStageBytes = kTileBytes + kVBytes;  // K then V
-  static constexpr int kStages = PT ? (HD == 64 ? 4 : 2) : (HD == 64 ? 3 : 2);
+  static constexpr int kVBytes = kWideV ? 2 * kKLoBytes : kKTileBytes;
+  static constexpr int kVTxBytes = kWideV ? 2 * kKLoBytes : kKTxBytes;
+  static constexpr int kStageBytes = kKTileBytes + kVBytes;  // K then V
+  static constexpr int kStages = PT ? (HD == 64 ? 4 : (kNarrowO ? 3 : 2)) : (HD == 64 ? 3 : 2);
   static constexpr int kQOff = 0;                          // [2 buffers][2 tiles]
   static constexpr int kKvOff = kQOff + 4 * kTileBytes;    // [stages][K, V]
   static constexpr int kPOff = kKvOff + kStages * kStageBytes;   // [2 tiles][2 k-blocks of 16 KB] (shared-memory P only)
@@ -66,18 +84,25 @@ struct AttnTcSmem {
   static constexpr int kBarOff = kOutOff + (kStagedOut ? 8 * 4096 : 0);
   static constexpr int kBytes = kBarOff + 512 + 1024;      // barriers + alignment slack
   static_assert(kBytes <= 232448, "exceeds the shared memory of an SM");
-  // TMEM columns: S_A [0,128) S_B [128,256) O_A [256,256+HD) O_B [256+HD', ...).  P in tensor memory: head_dim 64 has
-  // room for dedicated columns; head_dim 80 re-uses the first 64 columns of S (dead once the row sits in registers),
-  // which obliges the issuer to run P V before the next S.
+  static_assert(kKeys % 16 == 0 && kKeys % 8 == 0 && kKeys <= kTcTile, "key tile: whole UMMA k-steps and swizzle-atom rows");
+  static_assert(kStageBytes % 1024 == 0 && kTileBytes % 1024 == 0, "tiles start on swizzle-atom boundaries");
+  // TMEM columns: S_A [0, keys) S_B [keys, 2 keys), then O_A, O_B, then (if P has columns of its own) P_A, P_B.
+  // head_dim 64: 128 + 128 + 64 + 64 + 64 + 64 = 512.  head_dim 80 with 112 keys: 224 + 160 + 112 = 496.
+  // head_dim 80 with 128 keys: S 256 + O 2 x 128 (wide) = 512, and P re-uses the first 64 columns of S (dead once
+  // the row sits in registers), which obliges the issuer to run P V before the next S.
   // Dual-head units: an item whose query rows end in a single 128-row tile would leave warpgroup B idle for that
   // tile's whole key loop (c1: 577 tokens = 4.5 tiles, one unit in three).  With four K/V stages such tiles of TWO
   // adjacent heads form one unit instead: A works on head h, B on head h + 1, each with its own K/V tiles (two ring
   // stages per key tile).
   static constexpr bool kDualHeadOk = PT && HD == 64;   // the kernel's DUAL template argument may be set
-  static constexpr int kOCol0 = 256, kOStride = HD == 64 ? 64 : 128;
-  static constexpr bool kPAliasesS = PT && HD != 64;
-  static constexpr int kPCol0 = kPAliasesS ? 0 : 384, kPStride = kPAliasesS ? 128 : 64;
+  static constexpr int kSStride = kKeys;
+  static constexpr int kOCol0 = 2 * kKeys, kOStride = HD == 64 ? 64 : (kNarrowO ? HD : 128);
+  static constexpr bool kPAliasesS = PT && HD != 64 && !kNarrowO;
+  static constexpr int kPCol0 = kPAliasesS ? 0 : kOCol0 + 2 * kOStride, kPStride = kPAliasesS ? kSStride : kKeys / 2;
+  static_assert(kPAliasesS || !PT || kPCol0 + 2 * kPStride <= 512, "tensor memory columns");
+  static_assert(kOCol0 + 2 * kOStride <= 512, "tensor memory columns");
 };
+
 __device__ __forceinline__ void tmem_st_32x32_from(uint32_t taddr, const uint32_t* r) {
   asm volatile(
       "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
@@ -109,8 +134,35 @@ __device__ __forceinline__ void tmem_st_32x16(uint32_t taddr, const uint32_t (&r
 }
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
-template <int OFF>
-__device__ __forceinline__ void tmem_ld_32x32_at(uint32_t taddr, uint32_t (&r)[128]) {
+template <int OFF, int N>
+__device__ __forceinline__ void tmem_ld_32x16_at(uint32_t taddr, uint32_t (&r)[N]) {
+  static_assert(OFF + 16 <= N, "row buffer too short");
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=r"(r[OFF + 0]), "=r"(r[OFF + 1]), "=r"(r[OFF + 2]), "=r"(r[OFF + 3]), "=r"(r[OFF + 4]), "=r"(r[OFF + 5]),
+        "=r"(r[OFF + 6]), "=r"(r[OFF + 7]), "=r"(r[OFF + 8]), "=r"(r[OFF + 9]), "=r"(r[OFF + 10]), "=r"(r[OFF + 11]),
+        "=r"(r[OFF + 12]), "=r"(r[OFF + 13]), "=r"(r[OFF + 14]), "=r"(r[OFF + 15])
+      : "r"(taddr + OFF)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_st_32x16_from(uint32_t taddr, const uint32_t* r) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
+      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
+      ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+        "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
+      : "memory");
+}
+__device__ __forceinline__ void tmem_st_32x8_from(uint32_t taddr, const uint32_t* r) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+      ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7])
+      : "memory");
+}
+template <int OFF, int N>
+__device__ __forceinline__ void tmem_ld_32x32_at(uint32_t taddr, uint32_t (&r)[N]) {
+  static_assert(OFF + 32 <= N, "row buffer too short");
   asm volatile(
       "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
       "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
@@ -182,15 +234,16 @@ struct UnitInfo {
 // Unit order inside an item (the host's attention_schedule counts the same way).  Without dual-head units:
 // (head, pair of query tiles), the pair index fastest, the last pair possibly a single tile.  With them: first the
 // (head, FULL pair) units, then one unit per two heads for the odd last query tile.
-template <bool DUAL>
+template <bool DUAL, int KEYS>
 __device__ __forceinline__ UnitInfo decode_unit(const AttnTcParams& p, int unit, int& cursor) {
+  static_assert(!DUAL || KEYS == kTcTile, "dual-head units count query tiles as key tiles");
   int lo = cursor;
   while (lo + 1 < p.n_items && p.unit_prefix[lo + 1] <= unit) ++lo;
   cursor = lo;
   UnitInfo u;
   u.S = p.item_len[lo];
   u.row0 = p.item_start[lo];
-  u.n_kv = (u.S + kTcTile - 1) / kTcTile;
+  u.n_kv = (u.S + KEYS - 1) / KEYS;
   const int r = unit - p.unit_prefix[lo];
   if (DUAL) {
     const int full = u.n_kv >> 1;                  // query tiles == key tiles
@@ -264,7 +317,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_tc_kernel(const __grid_con
 
   auto q_tile = [&](int buf, int t) { return smem + L::kQOff + (buf * 2 + t) * L::kTileBytes; };
   auto k_tile = [&](int s) { return smem + L::kKvOff + s * L::kStageBytes; };
-  auto v_tile = [&](int s) { return smem + L::kKvOff + s * L::kStageBytes + L::kTileBytes; };
+  auto v_tile = [&](int s) { return smem + L::kKvOff + s * L::kStageBytes + L::kKTileBytes; };
   auto p_tile = [&](int w) { return smem + L::kPOff + w * 32768; };
 
   if (warp == 0) {
@@ -275,7 +328,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_tc_kernel(const __grid_con
       bool ok = true;
       int cursor = 0;
       for (int unit = blockIdx.x; unit < p.total_units && ok; unit += gridDim.x, ++u_cnt) {
-        const UnitInfo u = decode_unit<DUAL>(p, unit, cursor);
+        const UnitInfo u = decode_unit<DUAL, L::kKeys>(p, unit, cursor);
         const int qb = u_cnt & 1;
         if (!mbar_wait(&q_empty[qb], ((u_cnt >> 1) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
         mbar_expect_tx(&q_full[qb], u.n_q * L::kTileBytes);
@@ -291,14 +344,14 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_tc_kernel(const __grid_con
           const int xq = (u.head + (u.dual ? (jj & 1) : 0)) * HD;
           const int s = kv_it % NST;
           if (!mbar_wait(&kv_empty[s], ((kv_it / NST) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
-          const int y = static_cast<int>(u.row0) + j * kTcTile;
-          mbar_expect_tx(&k_full[s], L::kTileBytes);
-          tma_load_2d(k_tile(s), &p.map_lo, &k_full[s], p.d_model + xq, y);
-          if (HI) tma_load_2d(k_tile(s) + L::kLoBytes, &p.map_hi, &k_full[s], p.d_model + xq + 64, y);
-          mbar_expect_tx(&v_full[s], L::kVBytes);
-          tma_load_2d(v_tile(s), &p.map_lo, &v_full[s], 2 * p.d_model + xq, y);
-          if (L::kWideV) tma_load_2d(v_tile(s) + L::kLoBytes, &p.map_lo, &v_full[s], 2 * p.d_model + xq + 64, y);
-          else if (HI) tma_load_2d(v_tile(s) + L::kLoBytes, &p.map_hi, &v_full[s], 2 * p.d_model + xq + 64, y);
+          const int y = static_cast<int>(u.row0) + j * L::kKeys;
+          mbar_expect_tx(&k_full[s], L::kKTxBytes);
+          tma_load_2d(k_tile(s), &p.map_klo, &k_full[s], p.d_model + xq, y);
+          if (HI) tma_load_2d(k_tile(s) + L::kKLoBytes, &p.map_khi, &k_full[s], p.d_model + xq + 64, y);
+          mbar_expect_tx(&v_full[s], L::kVTxBytes);
+          tma_load_2d(v_tile(s), &p.map_klo, &v_full[s], 2 * p.d_model + xq, y);
+          if (L::kWideV) tma_load_2d(v_tile(s) + L::kKLoBytes, &p.map_klo, &v_full[s], 2 * p.d_model + xq + 64, y);
+          else if (HI) tma_load_2d(v_tile(s) + L::kKLoBytes, &p.map_khi, &v_full[s], 2 * p.d_model + xq + 64, y);
         }
       }
       if (!ok) {
@@ -310,10 +363,10 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_tc_kernel(const __grid_con
     // ------------------------------------------------------------------ UMMA issuer
     setmaxnreg_dec<kRegsLight>();
     if (lane == 0) {
-      constexpr uint32_t idesc_s = make_idesc_bf16(128, 128, 0, 0);     // S = Q K^T, both K-major
+      constexpr uint32_t idesc_s = make_idesc_bf16(128, L::kKeys, 0, 0);     // S = Q K^T, both K-major
       constexpr uint32_t idesc_o_lo = make_idesc_bf16(128, 64, 0, 1);   // O[:, 0:64] += P V, V is MN-major
       constexpr uint32_t idesc_o_hi = make_idesc_bf16(128, 16, 0, 1);   // O[:, 64:80]
-      constexpr uint32_t idesc_o_wide = make_idesc_bf16(128, 128, 0, 1); // O[:, 0:128] from the 128-column V tile
+      constexpr uint32_t idesc_o_wide = make_idesc_bf16(128, L::kNarrowO ? HD : 128, 0, 1); // O from the 128-column V tile
       uint32_t kv_it = 0, u_cnt = 0;
       uint32_t n_tiles[2] = {0, 0};            // S tiles issued per warpgroup (phase counters)
       uint32_t n_pv[2] = {0, 0};
@@ -324,12 +377,12 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_tc_kernel(const __grid_con
         const uint32_t ka = smem_u32(k_tile(s));
         const uint64_t ad = make_smem_desc(qa, 16, 1024, kSwizzle128B);
         const uint64_t bd = make_smem_desc(ka, 16, 1024, kSwizzle128B);
-        const uint32_t d = tmem_base + w * 128;
+        const uint32_t d = tmem_base + w * L::kSStride;
 #pragma unroll
         for (int k = 0; k < 4; ++k) umma_bf16_ss(d, ad + 2 * k, bd + 2 * k, idesc_s, k != 0);
         if (HI) {
           const uint64_t ah = make_smem_desc(qa + L::kLoBytes, 16, 256, kSwizzle32B);
-          const uint64_t bh = make_smem_desc(ka + L::kLoBytes, 16, 256, kSwizzle32B);
+          const uint64_t bh = make_smem_desc(ka + L::kKLoBytes, 16, 256, kSwizzle32B);
           umma_bf16_ss(d, ah, bh, idesc_s, 1);
         }
         umma_commit(&s_full[w]);
@@ -339,19 +392,19 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_tc_kernel(const __grid_con
         const uint32_t va = smem_u32(v_tile(s));
         const uint32_t d = tmem_base + L::kOCol0 + w * L::kOStride;
 #pragma unroll
-        for (int ks = 0; ks < 8; ++ks) {       // 16 keys per step
+        for (int ks = 0; ks < L::kKeys / 16; ++ks) {       // 16 keys per step
           const uint64_t bd = make_smem_desc(va + ks * 2048, 1024, 1024, kSwizzle128B);
           const uint32_t acc = (accumulate || ks != 0) ? 1u : 0u;
           if (L::kWideV) {
             // two 64-column swizzle atoms 16 KB apart (leading byte offset), 8-key groups 1 KB apart
             const uint32_t pt = tmem_base + L::kPCol0 + w * L::kPStride + ks * 8;
-            const uint64_t bw = make_smem_desc(va + ks * 2048, L::kLoBytes, 1024, kSwizzle128B);
+            const uint64_t bw = make_smem_desc(va + ks * 2048, L::kKLoBytes, 1024, kSwizzle128B);
             umma_bf16_ts(d, pt, bw, idesc_o_wide, acc);
           } else if (PT) {
             const uint32_t pt = tmem_base + L::kPCol0 + w * L::kPStride + ks * 8;   // 16 bf16 = 8 columns
             umma_bf16_ts(d, pt, bd, idesc_o_lo, acc);
             if (HI) {
-              const uint64_t bh = make_smem_desc(va + L::kLoBytes + ks * 512, 256, 256, kSwizzle32B);
+              const uint64_t bh = make_smem_desc(va + L::kKLoBytes + ks * 512, 256, 256, kSwizzle32B);
               umma_bf16_ts(d + 64, pt, bh, idesc_o_hi, acc);
             }
           } else {
@@ -359,7 +412,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_tc_kernel(const __grid_con
             const uint64_t ad = make_smem_desc(pa + (ks >> 2) * 16384 + (ks & 3) * 32, 16, 1024, kSwizzle128B);
             umma_bf16_ss(d, ad, bd, idesc_o_lo, acc);
             if (HI) {
-              const uint64_t bh = make_smem_desc(va + L::kLoBytes + ks * 512, 256, 256, kSwizzle32B);
+              const uint64_t bh = make_smem_desc(va + L::kKLoBytes + ks * 512, 256, 256, kSwizzle32B);
               umma_bf16_ss(d + 64, ad, bh, idesc_o_hi, acc);
             }
           }
@@ -370,12 +423,12 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_tc_kernel(const __grid_con
 
       bool pre_issued[2] = {false, false};       // S(w, 0) of this unit was already issued at the end of the previous one
       int cursor = 0;
-      UnitInfo un = decode_unit<DUAL>(p, min(static_cast<int>(blockIdx.x), p.total_units - 1), cursor);
+      UnitInfo un = decode_unit<DUAL, L::kKeys>(p, min(static_cast<int>(blockIdx.x), p.total_units - 1), cursor);
       for (int unit = blockIdx.x; unit < p.total_units && ok; unit += gridDim.x, ++u_cnt) {
         const UnitInfo u = un;
         const int qb = u_cnt & 1;
         const bool has_next = unit + static_cast<int>(gridDim.x) < p.total_units;
-        if (has_next) un = decode_unit<DUAL>(p, unit + gridDim.x, cursor);
+        if (has_next) un = decode_unit<DUAL, L::kKeys>(p, unit + gridDim.x, cursor);
         if (!mbar_wait(&q_full[qb], (u_cnt >> 1) & 1u, abort_flag)) { ok = false; break; }
         // K/V tile of warpgroup w at ring position kv_it: shared by both warpgroups, or (dual-head unit) one each
         const uint32_t step = 1 + u.dual;
@@ -450,7 +503,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_tc_kernel(const __grid_con
     const int quarter = warp & 3;                  // TMEM lane quarter of this warp
     const int row = quarter * 32 + lane;           // query row inside the tile == TMEM lane
     const uint32_t lane_addr = static_cast<uint32_t>(quarter * 32) << 16;
-    const uint32_t s_addr = tmem_base + lane_addr + w * 128;
+    const uint32_t s_addr = tmem_base + lane_addr + w * L::kSStride;
     const uint32_t o_addr = tmem_base + lane_addr + L::kOCol0 + w * L::kOStride;
     const uint32_t p_addr = tmem_base + lane_addr + L::kPCol0 + w * L::kPStride;
     uint8_t* p_row = p_tile(w) + row * 128;
@@ -515,13 +568,13 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_tc_kernel(const __grid_con
     };
 
     int cursor = 0;
-    UnitInfo u_next = decode_unit<DUAL>(p, min(static_cast<int>(blockIdx.x), p.total_units - 1), cursor);
+    UnitInfo u_next = decode_unit<DUAL, L::kKeys>(p, min(static_cast<int>(blockIdx.x), p.total_units - 1), cursor);
     for (int unit = blockIdx.x; unit < p.total_units && ok; unit += gridDim.x) {
       const UnitInfo u = u_next;
       ATTN_STAMP_PREV(10);
       const bool has_next = unit + static_cast<int>(gridDim.x) < p.total_units;
       if (w >= u.n_q) {                             // this warpgroup has no tile in the unit
-        if (has_next) u_next = decode_unit<DUAL>(p, unit + gridDim.x, cursor);
+        if (has_next) u_next = decode_unit<DUAL, L::kKeys>(p, unit + gridDim.x, cursor);
         if (pend && !flush_output()) { ok = false; break; }
         continue;
       }
@@ -534,23 +587,25 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_tc_kernel(const __grid_con
         if (!mbar_wait(&s_full[w], n & 1u, abort_flag)) { ok = false; break; }
         tc_fence_after_sync();
         ATTN_STAMP(1);
-        const int valid = min(kTcTile, u.S - j * kTcTile);     // keys of this tile that belong to the item
-        // the whole score row (128 fp32) in registers: four loads, one wait
-        uint32_t sr[128];
+        constexpr int KEYS = L::kKeys;
+        const int valid = min(KEYS, u.S - j * KEYS);           // keys of this tile that belong to the item
+        // the whole score row (one fp32 per key) in registers: a few loads, one wait
+        uint32_t sr[KEYS];
         __syncwarp();
         tmem_ld_32x32_at<0>(s_addr, sr);
         tmem_ld_32x32_at<32>(s_addr, sr);
         tmem_ld_32x32_at<64>(s_addr, sr);
-        tmem_ld_32x32_at<96>(s_addr, sr);
+        if constexpr (KEYS == 128) tmem_ld_32x32_at<96>(s_addr, sr); else tmem_ld_32x16_at<96>(s_addr, sr);
+        static_assert(KEYS == 128 || KEYS == 112, "score row: 4 x 32 columns, or 3 x 32 + 16");
         tmem_ld_wait();
         ATTN_STAMP(2);
-        if (valid < kTcTile) {                                  // last tile of the item: keys past its end
+        if (valid < KEYS) {                                     // last tile of the item: keys past its end
 #pragma unroll
-          for (int i = 0; i < 128; ++i) if (i >= valid) sr[i] = 0xff800000u;   // -inf
+          for (int i = 0; i < KEYS; ++i) if (i >= valid) sr[i] = 0xff800000u;   // -inf
         }
         float mx0 = -INFINITY, mx1 = -INFINITY;
 #pragma unroll
-        for (int i = 0; i < 128; i += 4) {
+        for (int i = 0; i < KEYS; i += 4) {
           mx0 = fmax3(mx0, __uint_as_float(sr[i]), __uint_as_float(sr[i + 1]));
           mx1 = fmax3(mx1, __uint_as_float(sr[i + 2]), __uint_as_float(sr[i + 3]));
         }
@@ -571,10 +626,10 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_tc_kernel(const __grid_con
         const uint64_t scale2 = pack2(p.scale_log2, p.scale_log2);
         const uint64_t nmb2 = pack2(-mb, -mb);
         // probabilities, kept packed in registers until the P buffer is free
-        uint32_t pk[64];
+        uint32_t pk[KEYS / 2];
         uint64_t acc0 = 0, acc1 = 0, acc2 = 0, acc3 = 0;       // (0.f, 0.f) pairs
 #pragma unroll
-        for (int i = 0; i < 64; i += 4) {
+        for (int i = 0; i < KEYS / 2; i += 4) {
 #pragma unroll
           for (int q = 0; q < 4; ++q) {
             const uint64_t t = ffma2(pack2(__uint_as_float(sr[2 * (i + q)]), __uint_as_float(sr[2 * (i + q) + 1])), scale2, nmb2);
@@ -620,11 +675,16 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_tc_kernel(const __grid_con
           }
           tmem_st_wait();
         }
-        if (PT) {
-          // P row into tensor memory: 128 bf16 = 64 columns of this thread's lane
+        if constexpr (PT) {
+          // P row into tensor memory: two bf16 per column of this thread's lane
           __syncwarp();
           tmem_st_32x32_from(p_addr, pk);
-          tmem_st_32x32_from(p_addr + 32, pk + 32);
+          if constexpr (KEYS == 128) {
+            tmem_st_32x32_from(p_addr + 32, pk + 32);
+          } else {
+            tmem_st_32x16_from(p_addr + 32, pk + 32);
+            tmem_st_32x8_from(p_addr + 48, pk + 48);
+          }
           tmem_st_wait();
         } else {
           // P row: 2 k-blocks of 64 keys, each row 128 bytes, 16-byte chunks XOR-swizzled by (row & 7)
@@ -641,7 +701,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_tc_kernel(const __grid_con
         if (lane == 0) mbar_arrive(&p_ready[w]);
         ATTN_STAMP(6);
         // decode the following unit here: the warp now waits for the issuer anyway
-        if (j == 0 && has_next) u_next = decode_unit<DUAL>(p, unit + gridDim.x, cursor);
+        if (j == 0 && has_next) u_next = decode_unit<DUAL, L::kKeys>(p, unit + gridDim.x, cursor);
       }
       if (!ok) break;
       pend = true;                                  // written later, see flush_output

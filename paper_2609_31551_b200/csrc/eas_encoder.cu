@@ -741,6 +741,12 @@ static eas_status launch_attention_tc(const bf16* qkv, bf16* out, const int32_t*
     EAS_TRY(make_tmap(&ap.map_lo, qkv, 2, dims, strides, box_lo, CU_TENSOR_MAP_SWIZZLE_128B));
     const uint32_t box_hi[2] = {16, kTcTile};
     EAS_TRY(make_tmap(&ap.map_hi, qkv, 2, dims, strides, box_hi, CU_TENSOR_MAP_SWIZZLE_32B));
+    // K and V tiles: the kernel's keys per tile (head_dim 80 with P in tensor memory: 112)
+    const uint32_t keys = hd == 64 ? AttnTcSmem<64, PT>::kKeys : AttnTcSmem<80, PT>::kKeys;
+    const uint32_t box_klo[2] = {64, keys};
+    EAS_TRY(make_tmap(&ap.map_klo, qkv, 2, dims, strides, box_klo, CU_TENSOR_MAP_SWIZZLE_128B));
+    const uint32_t box_khi[2] = {16, keys};
+    EAS_TRY(make_tmap(&ap.map_khi, qkv, 2, dims, strides, box_khi, CU_TENSOR_MAP_SWIZZLE_32B));
     const uint64_t odims[2] = {static_cast<uint64_t>(d), static_cast<uint64_t>(T)};
     const uint64_t ostrides[1] = {static_cast<uint64_t>(d) * 2};
     const uint32_t obox[2] = {64, 32};
