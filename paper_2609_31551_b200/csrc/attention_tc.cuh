@@ -9,7 +9,8 @@
 //
 //   warp 0       TMA producer: Q tiles (double buffered across units), K/V tiles through a ring
 //   warp 1       UMMA issuer:  S = Q K^T (128 x keys x {64|80}) into TMEM, O += P V (128 x {64|80} x keys) in TMEM;
-//                keys per K/V tile: 128 for head_dim 64, 112 for head_dim 80 (see AttnTcSmem)
+//                keys per K/V tile: 128 for head_dim 64, 112 for head_dim 80 (see AttnTcSmem); head_dim 80 has an
+//                issuer thread per warpgroup (warp 1 for tile A, warp 2 for tile B)
 //   warps 2, 3   idle (they complete the first warpgroup, whose registers are handed to the softmax warps)
 //   warps 4..7   softmax warpgroup of tile A: one thread per query row
 //   warps 8..11  softmax warpgroup of tile B
@@ -277,6 +278,11 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_tc_kernel(const __grid_con
   static_assert(!DUAL || L::kDualHeadOk, "dual-head units need four K/V stages and dedicated P columns");
   constexpr int HI = L::HI;
   constexpr int NST = L::kStages;
+  // head_dim 80: the single issuer thread (12 UMMAs per tile and warpgroup, about 90 cycles each) is what the softmax
+  // warpgroups wait for, so each warpgroup gets an issuer thread of its own (warps 1 and 2).  Not for head_dim 64: there
+  // the fixed order of one issuer keeps the two warpgroups' exponential phases apart, which is worth more.
+  constexpr bool kTwoIssuers = PT && HD != 64 && !L::kPAliasesS;
+  static_assert(!kTwoIssuers || (!DUAL && !L::kPAliasesS), "the two-issuer path has no dual-head units and needs dedicated P columns");
   extern __shared__ uint8_t smem_raw_attn[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw_attn) + 1023) & ~uintptr_t(1023));
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L::kBarOff);
@@ -288,17 +294,19 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_tc_kernel(const __grid_con
   uint64_t* s_full = bars + 4 + 3 * NST;   // [2]
   uint64_t* p_ready = s_full + 2;          // [2]
   uint64_t* pv_done = s_full + 4;          // [2]
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(s_full + 6);
+  uint64_t* s_free = s_full + 6;           // [2] two-issuer kernels: the warpgroup has read its scores out of tensor memory
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(s_full + 8);
   volatile uint32_t* abort_flag = tmem_slot + 1;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
   if (threadIdx.x == 0) {
+    // with one issuer thread per warpgroup both threads hand every K/V stage and Q buffer back
     for (int i = 0; i < 2; ++i) {
-      mbar_init(&q_full[i], 1); mbar_init(&q_empty[i], 1);
-      mbar_init(&s_full[i], 1); mbar_init(&p_ready[i], 4); mbar_init(&pv_done[i], 1);
+      mbar_init(&q_full[i], 1); mbar_init(&q_empty[i], kTwoIssuers ? 2 : 1);
+      mbar_init(&s_full[i], 1); mbar_init(&p_ready[i], 4); mbar_init(&pv_done[i], 1); mbar_init(&s_free[i], 4);
     }
-    for (int i = 0; i < NST; ++i) { mbar_init(&k_full[i], 1); mbar_init(&v_full[i], 1); mbar_init(&kv_empty[i], 1); }
+    for (int i = 0; i < NST; ++i) { mbar_init(&k_full[i], 1); mbar_init(&v_full[i], 1); mbar_init(&kv_empty[i], kTwoIssuers ? 2 : 1); }
     *abort_flag = 0;
     mbar_fence_init();
     tma_prefetch_desc(&p.map_lo);
@@ -359,8 +367,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_tc_kernel(const __grid_con
         while (clock64() - t0 < 4000000) {}     // let loads in flight land before the CTA retires
       }
     }
-  } else if (warp == 1) {
-    // ------------------------------------------------------------------ UMMA issuer
+  } else if (warp == 1 || (kTwoIssuers && warp == 2)) {
+    // ------------------------------------------------------------------ UMMA issuer(s)
     setmaxnreg_dec<kRegsLight>();
     if (lane == 0) {
       constexpr uint32_t idesc_s = make_idesc_bf16(128, L::kKeys, 0, 0);     // S = Q K^T, both K-major
@@ -421,77 +429,160 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_tc_kernel(const __grid_con
         ++n_pv[w];
       };
 
-      bool pre_issued[2] = {false, false};       // S(w, 0) of this unit was already issued at the end of the previous one
-      int cursor = 0;
-      UnitInfo un = decode_unit<DUAL, L::kKeys>(p, min(static_cast<int>(blockIdx.x), p.total_units - 1), cursor);
-      for (int unit = blockIdx.x; unit < p.total_units && ok; unit += gridDim.x, ++u_cnt) {
-        const UnitInfo u = un;
-        const int qb = u_cnt & 1;
-        const bool has_next = unit + static_cast<int>(gridDim.x) < p.total_units;
-        if (has_next) un = decode_unit<DUAL, L::kKeys>(p, unit + gridDim.x, cursor);
-        if (!mbar_wait(&q_full[qb], (u_cnt >> 1) & 1u, abort_flag)) { ok = false; break; }
-        // K/V tile of warpgroup w at ring position kv_it: shared by both warpgroups, or (dual-head unit) one each
-        const uint32_t step = 1 + u.dual;
-#pragma unroll
-        for (int w = 0; w < 2; ++w) {
-          if (w < u.n_q && !pre_issued[w]) {
-            const uint32_t g = kv_it + (u.dual ? w : 0);
-            if (!mbar_wait(&k_full[g % NST], (g / NST) & 1u, abort_flag)) { ok = false; break; }
-            tc_fence_after_sync();
-            issue_s(w, qb, g % NST);
+      if constexpr (kTwoIssuers) {
+        // One issuer thread per warpgroup (w = warp - 1), so every wait is in that warpgroup's own deterministic order:
+        //   S(next tile)  as soon as the warpgroup has read its previous scores out of tensor memory (s_free): the
+        //                 next scores are computed while the warpgroup works on the exponentials;
+        //   PV(tile)      when the warpgroup has stored P (p_ready).
+        // The thread walks EVERY tile of every unit of the CTA in order, also those of units its warpgroup has no part
+        // in: it waits until such a tile (or Q buffer) has landed and hands it back with a plain arrival, so that both
+        // issuers see every phase of every barrier and a parity can never be mistaken for an earlier phase.
+        const int w = warp - 1;
+        struct Pos {                                 // a tile position in the CTA's sequence, with its unit's facts
+          int unit, j, n_kv, hint;
+          uint32_t ucnt, g;                          // units before it (Q buffer), tiles before it (ring stage)
+          bool active, end;
+        };
+        auto enter_unit = [&](Pos& c) {              // c.unit / c.ucnt / c.g are set; fills the unit's facts
+          if (c.unit >= p.total_units) { c.end = true; return; }
+          const UnitInfo u = decode_unit<DUAL, L::kKeys>(p, c.unit, c.hint);
+          c.n_kv = u.n_kv;
+          c.active = w < u.n_q;
+          c.j = 0;
+        };
+        auto next_tile = [&](Pos& c) {
+          ++c.j; ++c.g;
+          if (c.j >= c.n_kv) { c.unit += gridDim.x; ++c.ucnt; enter_unit(c); }
+        };
+        Pos pc;                                      // in-order position: every tile is visited
+        pc.unit = blockIdx.x; pc.ucnt = 0; pc.g = 0; pc.hint = 0; pc.end = false;
+        enter_unit(pc);
+        bool s_issued = false;                       // S of the own tile at pc is already in flight
+        uint32_t q_seen = 0;                         // units before this one have had their Q seen landing by this thread
+        while (!pc.end && ok) {
+          const int qb = pc.ucnt & 1;
+          if (pc.j == 0) {                           // entering a unit: see its Q land; hand it back at once if unused
+            if (pc.ucnt >= q_seen) {                 // (a look-ahead S may have seen it already, and handed it back)
+              if (!mbar_wait(&q_full[qb], (pc.ucnt >> 1) & 1u, abort_flag)) { ok = false; break; }
+              q_seen = pc.ucnt + 1;
+            }
+            if (!pc.active) mbar_arrive(&q_empty[qb]);
           }
+          const int s = pc.g % NST;
+          const uint32_t ph = (pc.g / NST) & 1u;
+          if (!pc.active) {
+            if (!mbar_wait(&k_full[s], ph, abort_flag) || !mbar_wait(&v_full[s], ph, abort_flag)) { ok = false; break; }
+            mbar_arrive(&kv_empty[s]);
+            next_tile(pc);
+            continue;
+          }
+          if (!s_issued) {                           // first own tile, or the look-ahead below was not possible
+            if (!mbar_wait(&k_full[s], ph, abort_flag)) { ok = false; break; }
+            tc_fence_after_sync();
+            issue_s(w, qb, s);
+            if (pc.j + 1 >= pc.n_kv) umma_commit(&q_empty[qb]);
+          }
+          s_issued = false;
+          // the next own tile, if it is close enough that its barriers' previous phases have been seen by this thread
+          // (strictly inside the ring: the stage of tile pc.g + NST is the one this thread still holds)
+          Pos nx = pc;
+          next_tile(nx);
+          while (!nx.end && !nx.active && nx.g - pc.g + 1 < static_cast<uint32_t>(NST) && nx.ucnt <= pc.ucnt + 1) next_tile(nx);
+          const bool ahead = !nx.end && nx.active && nx.g - pc.g < static_cast<uint32_t>(NST) && nx.ucnt <= pc.ucnt + 1;
+          if (ahead) {
+            if (!mbar_wait(&s_free[w], (n_tiles[w] - 1) & 1u, abort_flag)) { ok = false; break; }
+            const int nqb = nx.ucnt & 1;
+            if (nx.ucnt >= q_seen) {
+              if (!mbar_wait(&q_full[nqb], (nx.ucnt >> 1) & 1u, abort_flag)) { ok = false; break; }
+              q_seen = nx.ucnt + 1;
+            }
+            const int sn = nx.g % NST;
+            if (!mbar_wait(&k_full[sn], (nx.g / NST) & 1u, abort_flag)) { ok = false; break; }
+            tc_fence_after_sync();
+            issue_s(w, nqb, sn);
+            if (nx.j + 1 >= nx.n_kv) umma_commit(&q_empty[nqb]);
+            s_issued = true;
+          }
+          if (!mbar_wait(&p_ready[w], n_pv[w] & 1u, abort_flag)) { ok = false; break; }
+          if (!mbar_wait(&v_full[s], ph, abort_flag)) { ok = false; break; }
+          tc_fence_after_sync();
+          issue_pv(w, s, pc.j != 0);
+          umma_commit(&kv_empty[s]);                 // arrives when everything this thread has issued so far is complete
+          next_tile(pc);
         }
-        if (!ok) break;
-        pre_issued[0] = pre_issued[1] = false;
-        bool next_q_ready = false;
-        const int n_kv = u.n_kv, n_q = u.n_q, next_n_q = un.n_q;
-        const uint32_t b_off = u.dual ? 1u : 0u, b_off_next = un.dual ? 1u : 0u;   // B's tile relative to A's
-        for (int j = 0; j < n_kv && ok; ++j, kv_it += step) {
-          const bool last = j + 1 == n_kv;
+      } else {
+        bool pre_issued[2] = {false, false};       // S(w, 0) of this unit was already issued at the end of the previous one
+        int cursor = 0;
+        UnitInfo un = decode_unit<DUAL, L::kKeys>(p, min(static_cast<int>(blockIdx.x), p.total_units - 1), cursor);
+        for (int unit = blockIdx.x; unit < p.total_units && ok; unit += gridDim.x, ++u_cnt) {
+          const UnitInfo u = un;
+          const int qb = u_cnt & 1;
+          const bool has_next = unit + static_cast<int>(gridDim.x) < p.total_units;
+          if (has_next) un = decode_unit<DUAL, L::kKeys>(p, unit + gridDim.x, cursor);
+          if (!mbar_wait(&q_full[qb], (u_cnt >> 1) & 1u, abort_flag)) { ok = false; break; }
+          // K/V tile of warpgroup w at ring position kv_it: shared by both warpgroups, or (dual-head unit) one each
+          const uint32_t step = 1 + u.dual;
 #pragma unroll
           for (int w = 0; w < 2; ++w) {
-            if (w >= n_q) break;
-            const uint32_t g = kv_it + (w ? b_off : 0u);                                          // this tile
-            const uint32_t gn = kv_it + step + (w ? (last ? b_off_next : b_off) : 0u);            // the warpgroup's next one
-            const int s = g % NST, sn = gn % NST;
-            // warpgroup B shares A's tiles unless the unit is dual-head: A has already seen them land
-            const bool own_tile = w == 0 || (b_off | (last ? b_off_next : 0u)) != 0u;
-            // P(w, j) is in shared memory, S(w) has been read, O(w) has been rescaled if it had to be
-            if (!mbar_wait(&p_ready[w], (n_pv[w]) & 1u, abort_flag)) { ok = false; break; }
-            tc_fence_after_sync();
-            // next scores first (the softmax of the next tile overlaps P V of this one); after the unit's last
-            // tile the next scores are the first tile of the NEXT unit, so the pipeline never drains
-            // next scores before P V, so that the next softmax overlaps it -- unless P re-uses S's columns
-            if (!last && !L::kPAliasesS) {
-              if (own_tile && !mbar_wait(&k_full[sn], (gn / NST) & 1u, abort_flag)) { ok = false; break; }
+            if (w < u.n_q && !pre_issued[w]) {
+              const uint32_t g = kv_it + (u.dual ? w : 0);
+              if (!mbar_wait(&k_full[g % NST], (g / NST) & 1u, abort_flag)) { ok = false; break; }
               tc_fence_after_sync();
-              issue_s(w, qb, sn);
+              issue_s(w, qb, g % NST);
             }
-            if (own_tile && !mbar_wait(&v_full[s], (g / NST) & 1u, abort_flag)) { ok = false; break; }
-            tc_fence_after_sync();
-            issue_pv(w, s, j != 0);
-            if (!last && L::kPAliasesS) {
-              if (own_tile && !mbar_wait(&k_full[sn], (gn / NST) & 1u, abort_flag)) { ok = false; break; }
-              tc_fence_after_sync();
-              issue_s(w, qb, sn);
-            }
-            if (last && has_next && w < next_n_q) {
-              // the unit's output is waiting for this P V, so it went first; now the first scores of the next unit
-              if (!next_q_ready) {
-                if (!mbar_wait(&q_full[qb ^ 1], ((u_cnt + 1) >> 1) & 1u, abort_flag)) { ok = false; break; }
-                next_q_ready = true;
-              }
-              if (own_tile && !mbar_wait(&k_full[sn], (gn / NST) & 1u, abort_flag)) { ok = false; break; }
-              tc_fence_after_sync();
-              issue_s(w, qb ^ 1, sn);
-              pre_issued[w] = true;
-            }
-            // K and V of this tile are free once everything issued so far completes: after the last warpgroup that
-            // uses them
-            if (b_off != 0u || w + 1 == n_q) umma_commit(&kv_empty[s]);
           }
+          if (!ok) break;
+          pre_issued[0] = pre_issued[1] = false;
+          bool next_q_ready = false;
+          const int n_kv = u.n_kv, n_q = u.n_q, next_n_q = un.n_q;
+          const uint32_t b_off = u.dual ? 1u : 0u, b_off_next = un.dual ? 1u : 0u;   // B's tile relative to A's
+          for (int j = 0; j < n_kv && ok; ++j, kv_it += step) {
+            const bool last = j + 1 == n_kv;
+#pragma unroll
+            for (int w = 0; w < 2; ++w) {
+              if (w >= n_q) break;
+              const uint32_t g = kv_it + (w ? b_off : 0u);                                          // this tile
+              const uint32_t gn = kv_it + step + (w ? (last ? b_off_next : b_off) : 0u);            // the warpgroup's next one
+              const int s = g % NST, sn = gn % NST;
+              // warpgroup B shares A's tiles unless the unit is dual-head: A has already seen them land
+              const bool own_tile = w == 0 || (b_off | (last ? b_off_next : 0u)) != 0u;
+              // P(w, j) is in shared memory, S(w) has been read, O(w) has been rescaled if it had to be
+              if (!mbar_wait(&p_ready[w], (n_pv[w]) & 1u, abort_flag)) { ok = false; break; }
+              tc_fence_after_sync();
+              // next scores first (the softmax of the next tile overlaps P V of this one); after the unit's last
+              // tile the next scores are the first tile of the NEXT unit, so the pipeline never drains
+              // next scores before P V, so that the next softmax overlaps it -- unless P re-uses S's columns
+              if (!last && !L::kPAliasesS) {
+                if (own_tile && !mbar_wait(&k_full[sn], (gn / NST) & 1u, abort_flag)) { ok = false; break; }
+                tc_fence_after_sync();
+                issue_s(w, qb, sn);
+              }
+              if (own_tile && !mbar_wait(&v_full[s], (g / NST) & 1u, abort_flag)) { ok = false; break; }
+              tc_fence_after_sync();
+              issue_pv(w, s, j != 0);
+              if (!last && L::kPAliasesS) {
+                if (own_tile && !mbar_wait(&k_full[sn], (gn / NST) & 1u, abort_flag)) { ok = false; break; }
+                tc_fence_after_sync();
+                issue_s(w, qb, sn);
+              }
+              if (last && has_next && w < next_n_q) {
+                // the unit's output is waiting for this P V, so it went first; now the first scores of the next unit
+                if (!next_q_ready) {
+                  if (!mbar_wait(&q_full[qb ^ 1], ((u_cnt + 1) >> 1) & 1u, abort_flag)) { ok = false; break; }
+                  next_q_ready = true;
+                }
+                if (own_tile && !mbar_wait(&k_full[sn], (gn / NST) & 1u, abort_flag)) { ok = false; break; }
+                tc_fence_after_sync();
+                issue_s(w, qb ^ 1, sn);
+                pre_issued[w] = true;
+              }
+              // K and V of this tile are free once everything issued so far completes: after the last warpgroup that
+              // uses them
+              if (b_off != 0u || w + 1 == n_q) umma_commit(&kv_empty[s]);
+            }
+          }
+          if (ok) umma_commit(&q_empty[qb]);
         }
-        if (ok) umma_commit(&q_empty[qb]);
       }
     }
   } else if (warp < 4) {
@@ -598,6 +689,11 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_tc_kernel(const __grid_con
         if constexpr (KEYS == 128) tmem_ld_32x32_at<96>(s_addr, sr); else tmem_ld_32x16_at<96>(s_addr, sr);
         static_assert(KEYS == 128 || KEYS == 112, "score row: 4 x 32 columns, or 3 x 32 + 16");
         tmem_ld_wait();
+        if constexpr (kTwoIssuers) {      // the scores are in registers: the issuer may start the next S into these columns
+          tc_fence_before_sync();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&s_free[w]);
+        }
         ATTN_STAMP(2);
         if (valid < KEYS) {                                     // last tile of the item: keys past its end
 #pragma unroll
