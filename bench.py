@@ -124,6 +124,26 @@ def measured_peaks():
     return dict(hbm=6650.0, burst=1590.0, sustained=1400.0, source="fallback")
 
 
+def other_rooflines(cfg, shapes, f, acc, n_prof, peaks):
+    """The two other kernel classes of a step against their own roofs (start-to-start times, so launch gaps count):
+    attention against the sustained bf16 tensor peak (its exponentials, not the tensor pipe, pace it), and the norm
+    kernels against the measured HBM copy rate with 6 algorithmic bytes per element (fp32 in, bf16 out)."""
+    out = []
+    if 5 in acc and acc[5][0] > 0:
+        t = acc[5][0] / n_prof * 1e-3
+        tf = f["attention"] / t / 1e12
+        out.append({"kernel": "attn_tc_kernel", "bound": "tensor", "achieved": tf, "peak": peaks["sustained"], "unit": "TFLOP/s",
+                    "frac": tf / peaks["sustained"], "launches_per_step": acc[5][1] // n_prof})
+    if 3 in acc and acc[3][0] > 0:
+        t = acc[3][0] / n_prof * 1e-3
+        n_norm = acc[3][1] // n_prof
+        gbs = 6.0 * f["tokens"] * cfg["d_model"] * n_norm / t / 1e9
+        out.append({"kernel": "norm_kernel", "bound": "hbm", "achieved": gbs, "peak": peaks["hbm"], "unit": "GB/s",
+                    "frac": gbs / peaks["hbm"], "launches_per_step": n_norm,
+                    "note": "6 bytes per element and launch; head and embed norms touch fewer rows, so this is an upper bound on bytes"})
+    return out
+
+
 def workload(cfg_name, mb, seed_shift=0):
     cfg = S.get_config(cfg_name)
     ci = S.configs.CONFIG_INDEX[cfg_name]
@@ -322,6 +342,7 @@ def run_cuda(args):
                          "traffic": 144.2e6 if (args.config == "c1" and args.micro_batch == 32) else None,
                          "traffic_note": "dram read+write bytes of one fc1 GEMM launch (ncu); algorithmic 197.5e6",
                          "launches_per_step": gemm_launch, "avg_launch_ms": gemm_ms / max(gemm_launch, 1)},
+            "roofline_other": other_rooflines(cfg, shapes, f, acc, n_prof, peaks),
             "kernel_breakdown": breakdown,
         }
         if world == 1 and not args.no_cpu_baseline:
