@@ -151,3 +151,31 @@ def test_attention_dual_head_units(H):
         assert torch.equal(out, out2), budget
     out3, _ = P.kernel_attention(_dev(qkv), cu, H, hd, impl=1)
     assert (out.float() - out3.float()).abs().max() <= 2e-2
+
+
+@pytest.mark.parametrize("H", [1, 3])
+def test_attention_head_dim_80_key_tile_edges(H):
+    """head_dim 80 runs on 112-key tiles with one issuer thread per warpgroup: item lengths around the multiples of 112
+    and of 128 (query tiles stay 128 rows), single-tile items whose second warpgroup idles, and few CTAs for many units
+    (long per-CTA unit sequences, look-ahead across unit boundaries)."""
+    import paper_2609_31551_b200 as P
+    hd, lens = 80, [112, 113, 224, 225, 336, 1, 127, 128, 129, 257, 640, 1000, 16, 111]
+    rng = np.random.Generator(np.random.PCG64(1200 + H))
+    T, d = sum(lens), H * hd
+    qkv = _bf16_exact(rng, (T, 3 * d))
+    qkv[:, : 2 * d] *= 1.5
+    qkv = S.round_to_bf16(qkv)
+    cu = np.concatenate([[0], np.cumsum(lens)]).astype(np.int32)
+    q = O._t(qkv)
+    ref = torch.cat([O.attention_one_item(q[a:b, :d].reshape(-1, H, hd), q[a:b, d:2 * d].reshape(-1, H, hd),
+                                          q[a:b, 2 * d:].reshape(-1, H, hd)) for a, b in zip(cu[:-1], cu[1:])])
+    out, status = P.kernel_attention(_dev(qkv), cu, H, hd, impl=0)
+    torch.cuda.synchronize()
+    assert int(status[0]) == 0
+    err = (out.double().cpu() - ref).abs()
+    assert err.max() <= 2e-2, (err.max(), np.unravel_index(int(err.argmax()), err.shape))
+    for budget in (1, 2, 5, 37):
+        out2, st2 = P.kernel_attention(_dev(qkv), cu, H, hd, impl=0, sm_budget=budget)
+        torch.cuda.synchronize()
+        assert int(st2[0]) == 0
+        assert torch.equal(out, out2), budget
