@@ -1,14 +1,18 @@
 // Persistent bf16 GEMM for sm_100a:  D[M,N] = A[M,K] * W[N,K]^T  with a fused epilogue.
 //
-//   warp 0, 10  TMA producers (A tiles, W tiles): 128x64 A tiles and 256x64 W tiles into a shared-memory ring
-//   warp 1      UMMA issuer: tcgen05.mma 128x256x16, fp32 accumulators in TMEM, two accumulator
-//               buffers (2 x 256 columns) so that the epilogue of tile i overlaps the main loop of tile i+1
+//   warp 0, 10  TMA producers, one thread per operand (A tiles in warp 0, W tiles in warp 10) into a shared-memory ring
+//   warp 1      UMMA issuer: tcgen05.mma (128x256x16, or 256x256x16 for a CTA pair), fp32 accumulators in TMEM, two
+//               accumulator buffers (2 x 256 columns) so that the epilogue of tile i overlaps the main loop of tile i+1
 //   warps 2..9  epilogue: tcgen05.ld -> bias / activation / rotary -> swizzled shared-memory staging -> TMA store
 //               (TMA reduce-add into the fp32 residual stream); scatter epilogues (row maps) store directly
 //
+// Three tile shapes (template arguments CTAS, NW, KD; the launcher picks by estimated time): one CTA per 128x256 tile,
+// a CTA pair (cta_group::2) per 256x256 tile with "deep" stages, a pair per "wide" 256x512 tile.
+//
 // The grid is `sm_budget` CTAs (one per SM: the shared-memory request excludes a second resident
-// CTA) and each CTA walks tiles  blockIdx.x, blockIdx.x + gridDim.x, ...  in a fixed order, so the
-// result never depends on the budget: no split-K, no atomics.
+// CTA) and each CTA walks tiles  blockIdx.x, blockIdx.x + gridDim.x, ...  in a fixed order; every output element is
+// accumulated over K in the same order whatever the tile shape, so the result never depends on the budget: no split-K,
+// no atomics on the accumulation (the fp32 residual update is one add per element).
 #pragma once
 #include "ptx.cuh"
 
@@ -22,8 +26,8 @@ constexpr int kABytes = kBM * kBK * 2;            // 16 KB: 128 rows of A
 // one CTA per tile: a stage holds A (16 KB) + the whole 256-row weight tile (32 KB), 4 stages;
 // CTA pair per 256x256 tile: a stage holds A (16 KB) + this CTA's 128 weight rows (16 KB), 6 stages
 // NW = 2 ("wide", CTA pairs only): the pair owns a 256x512 tile, i.e. two 256-column accumulators fed by the same
-// A tile.  That cuts the operand bytes per FLOP by a quarter (the L2 -> SM path is what bounds the main loop) at the
-// price of a single accumulator set: the epilogue no longer overlaps the next main loop, so it pays for large K only.
+// A tile (three TMA operations for twice the columns) at the price of a single accumulator set: the epilogue no longer
+// overlaps the next main loop, so it pays for large K only.
 // KD = 2 ("deep"): a stage holds TWO 64-wide k-blocks of each operand, fetched by ONE TMA operation per operand
 // (a 3-D box {64 columns, rows, 2 k-blocks}, which lands as two consecutive swizzle-atom blocks).  Measured on B200:
 // what a CTA can pull from L2 is set by the number of TMA operations in flight, not by their bytes (two 16 KB
