@@ -291,13 +291,29 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_kernel(const __grid_cons
           if (p.rope_cs != nullptr && col0 < p.rope_ncols && arow < p.M) {
             const float2* cs = p.rope_cs + static_cast<long long>(arow) * p.rope_pairs;
             int pi = (col0 % p.head_dim) >> 1;
+            if ((p.rope_pairs & 1) == 0 && (pi & 1) == 0) {
+              // two (cos, sin) pairs per 16-byte load: the row's table is 16-byte aligned and wraps at an even index
+              const float4* cs4 = reinterpret_cast<const float4*>(cs);
 #pragma unroll
-            for (int j = 0; j < 16; ++j) {
-              const float2 t = __ldg(cs + pi);
-              const float x0 = v[2 * j], x1 = v[2 * j + 1];
-              v[2 * j] = x0 * t.x - x1 * t.y;
-              v[2 * j + 1] = x1 * t.x + x0 * t.y;
-              if (++pi == p.rope_pairs) pi = 0;
+              for (int j = 0; j < 16; j += 2) {
+                const float4 t = __ldg(cs4 + (pi >> 1));
+                const float x0 = v[2 * j], x1 = v[2 * j + 1], x2 = v[2 * j + 2], x3 = v[2 * j + 3];
+                v[2 * j] = x0 * t.x - x1 * t.y;
+                v[2 * j + 1] = x1 * t.x + x0 * t.y;
+                v[2 * j + 2] = x2 * t.z - x3 * t.w;
+                v[2 * j + 3] = x3 * t.z + x2 * t.w;
+                pi += 2;
+                if (pi == p.rope_pairs) pi = 0;
+              }
+            } else {
+#pragma unroll
+              for (int j = 0; j < 16; ++j) {
+                const float2 t = __ldg(cs + pi);
+                const float x0 = v[2 * j], x1 = v[2 * j + 1];
+                v[2 * j] = x0 * t.x - x1 * t.y;
+                v[2 * j + 1] = x1 * t.x + x0 * t.y;
+                if (++pi == p.rope_pairs) pi = 0;
+              }
             }
           }
           if (ACT == ACT_GELU) {
