@@ -577,6 +577,7 @@ struct GemmCall {
   const int* pos_idx = nullptr;
   const bf16* pos = nullptr;
   const float2* rope_cs = nullptr;
+  long long rope_stride = 0;   // rows of the [pair][row] table
   int rope_pairs = 0, rope_ncols = 0, head_dim = 0;
 };
 }  // namespace
@@ -634,7 +635,7 @@ static eas_status launch_gemm(const GemmCall& g, int budget, cudaStream_t stream
   p.bias = L.b;
   p.out = g.out; p.ldo = g.ldo; p.resid = g.resid;
   p.row_map = g.row_map; p.pos_idx = g.pos_idx; p.pos = g.pos;
-  p.rope_cs = g.rope_cs; p.rope_pairs = g.rope_pairs; p.rope_ncols = g.rope_ncols; p.head_dim = g.head_dim > 0 ? g.head_dim : 64;
+  p.rope_cs = g.rope_cs; p.rope_stride = g.rope_stride; p.rope_pairs = g.rope_pairs; p.rope_ncols = g.rope_ncols; p.head_dim = g.head_dim > 0 ? g.head_dim : 64;
   p.status = status;
   // TMA-store epilogue whenever output rows are the A rows and any residual is accumulated in place
   p.use_tma_out = tma_out ? 1 : 0;
@@ -944,7 +945,7 @@ static eas_status encode_impl(eas_encoder* e, const eas_packed_inputs* in, void*
       GemmCall g;
       g.A = nbuf; g.a_run = d; g.a_row_elems = d; g.a_rows = T; g.M = static_cast<int>(T); g.lin = &L.qkv;
       g.out = qkv; g.ldo = 3LL * d;
-      if (c.pos == EAS_POS_ROPE_2D) { g.rope_cs = rope; g.rope_pairs = e->hd / 2; g.rope_ncols = 2 * d; g.head_dim = e->hd; }
+      if (c.pos == EAS_POS_ROPE_2D) { g.rope_cs = rope; g.rope_stride = T; g.rope_pairs = e->hd / 2; g.rope_ncols = 2 * d; g.head_dim = e->hd; }
       EAS_TRY(mark(e, EAS_KC_GEMM_QKV, stream));
       EAS_TRY(launch_gemm(g, budget, stream, status)); ++launches;
     }

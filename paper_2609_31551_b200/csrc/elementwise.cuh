@@ -185,7 +185,7 @@ struct PrepParams {
   int* embed_row_map;     // [n_embed_rows] -> residual-stream row or -1
   int* embed_pos_idx;     // [n_embed_rows] -> position-table row
   int* head_src_rows;     // [out rows] (MLP projector: tokens without CLS)
-  float2* rope_cs;        // [total_tokens, rope_pairs]
+  float2* rope_cs;        // [rope_pairs][total_tokens]: the GEMM epilogue's 32 rows of a warp read consecutive entries
   float* x;               // residual stream (CLS rows are written here)
   const bf16* cls;        // [d]
   const bf16* pos;        // [max_pos, d]
@@ -246,7 +246,7 @@ __global__ void __launch_bounds__(256) prep_kernel(const __grid_constant__ PrepP
       const float ang = static_cast<float>(i < nf ? r : c) * freq;
       float sn, cs;
       sincosf(ang, &sn, &cs);
-      p.rope_cs[idx] = make_float2(cs, sn);
+      p.rope_cs[static_cast<long long>(i) * p.total_tokens + tok] = make_float2(cs, sn);   // [pair][token]
     }
   }
   if (p.family == 2) {

@@ -68,7 +68,9 @@ struct alignas(64) GemmParams {
   const int* row_map;     // optional: output row of each A row, negative = drop the row
   const int* pos_idx;     // optional (with pos): row of the position table added to each A row
   const bf16* pos;        // optional position table [*, N]
-  const float2* rope_cs;  // optional (cos, sin) per (A row, pair): columns < rope_ncols are rotated as adjacent pairs
+  const float2* rope_cs;  // optional (cos, sin), stored [pair][A row] so that the 32 rows of a warp read consecutive
+                          // entries: columns < rope_ncols are rotated as adjacent pairs
+  long long rope_stride;  // entries per pair (= rows of the table)
   int rope_pairs;         // pairs per head (head_dim / 2)
   int rope_ncols;         // rotate output columns [0, rope_ncols)
   int head_dim;
@@ -289,31 +291,15 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_kernel(const __grid_cons
             v[4 * q] += b.x; v[4 * q + 1] += b.y; v[4 * q + 2] += b.z; v[4 * q + 3] += b.w;
           }
           if (p.rope_cs != nullptr && col0 < p.rope_ncols && arow < p.M) {
-            const float2* cs = p.rope_cs + static_cast<long long>(arow) * p.rope_pairs;
             int pi = (col0 % p.head_dim) >> 1;
-            if ((p.rope_pairs & 1) == 0 && (pi & 1) == 0) {
-              // two (cos, sin) pairs per 16-byte load: the row's table is 16-byte aligned and wraps at an even index
-              const float4* cs4 = reinterpret_cast<const float4*>(cs);
+            const float2* cs = p.rope_cs + arow;
 #pragma unroll
-              for (int j = 0; j < 16; j += 2) {
-                const float4 t = __ldg(cs4 + (pi >> 1));
-                const float x0 = v[2 * j], x1 = v[2 * j + 1], x2 = v[2 * j + 2], x3 = v[2 * j + 3];
-                v[2 * j] = x0 * t.x - x1 * t.y;
-                v[2 * j + 1] = x1 * t.x + x0 * t.y;
-                v[2 * j + 2] = x2 * t.z - x3 * t.w;
-                v[2 * j + 3] = x3 * t.z + x2 * t.w;
-                pi += 2;
-                if (pi == p.rope_pairs) pi = 0;
-              }
-            } else {
-#pragma unroll
-              for (int j = 0; j < 16; ++j) {
-                const float2 t = __ldg(cs + pi);
-                const float x0 = v[2 * j], x1 = v[2 * j + 1];
-                v[2 * j] = x0 * t.x - x1 * t.y;
-                v[2 * j + 1] = x1 * t.x + x0 * t.y;
-                if (++pi == p.rope_pairs) pi = 0;
-              }
+            for (int j = 0; j < 16; ++j) {
+              const float2 t = __ldg(cs + pi * p.rope_stride);
+              const float x0 = v[2 * j], x1 = v[2 * j + 1];
+              v[2 * j] = x0 * t.x - x1 * t.y;
+              v[2 * j + 1] = x1 * t.x + x0 * t.y;
+              if (++pi == p.rope_pairs) pi = 0;
             }
           }
           if (ACT == ACT_GELU) {
@@ -467,11 +453,11 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_kernel(const __grid_cons
         if (p.rope_cs != nullptr && col0 < p.rope_ncols) {
           // rotary: adjacent columns (2i, 2i+1) of a head form pair i (the weight rows were
           // re-ordered at create time so that the two halves of a pair sit side by side)
-          const float2* cs = p.rope_cs + static_cast<long long>(arow) * p.rope_pairs;
+          const float2* cs = p.rope_cs + arow;
           int pi = (col0 % p.head_dim) >> 1;
 #pragma unroll
           for (int j = 0; j < 16; ++j) {
-            const float2 t = __ldg(cs + pi);
+            const float2 t = __ldg(cs + pi * p.rope_stride);
             const float x0 = v[2 * j], x1 = v[2 * j + 1];
             v[2 * j] = x0 * t.x - x1 * t.y;
             v[2 * j + 1] = x1 * t.x + x0 * t.y;
