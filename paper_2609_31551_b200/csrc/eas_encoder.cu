@@ -577,6 +577,7 @@ struct GemmCall {
   const int* pos_idx = nullptr;
   const bf16* pos = nullptr;
   const float2* rope_cs = nullptr;
+  int reverse = 0;             // walk the tiles last to first
   long long rope_stride = 0;   // rows of the [pair][row] table
   int rope_pairs = 0, rope_ncols = 0, head_dim = 0;
 };
@@ -630,6 +631,7 @@ static eas_status launch_gemm(const GemmCall& g, int budget, cudaStream_t stream
   p.kb_per_tap = static_cast<int>(g.a_run / kBK);
   p.k_blocks = deep ? (p.kb_per_tap + 1) / 2 : p.kb_per_tap * g.taps;
   p.conv_stride = g.conv_stride;
+  p.reverse = g.reverse;
   p.m_blocks = (g.M + kBM * ctas - 1) / (kBM * ctas);
   p.n_blocks = (L.N + tile_n - 1) / tile_n;
   p.bias = L.b;
@@ -685,10 +687,11 @@ static eas_status launch_norm(int kind, bool out_fp32, const NormParams& p, int 
 // schedule order: longest items first (stable), so the tail of the static round-robin is short work
 // dual_head: the tcgen05 kernel's unit order for head_dim 64 (see decode_unit): per item H x (full pairs of query
 // tiles), then one unit per two heads for an odd last tile.
+// reverse: items of equal length are taken last to first (the producer of qkv wrote the last rows most recently: L2).
 static void attention_schedule(const int32_t* cu, int n_items, int rows_per_unit, int H, int* item_start, int* item_len,
-                               int* unit_prefix, int* total_units, bool dual_head = false) {
+                               int* unit_prefix, int* total_units, bool dual_head = false, bool reverse = false) {
   std::vector<int> order(n_items);
-  for (int i = 0; i < n_items; ++i) order[i] = i;
+  for (int i = 0; i < n_items; ++i) order[i] = reverse ? n_items - 1 - i : i;
   std::stable_sort(order.begin(), order.end(), [&](int a, int b) { return (cu[a + 1] - cu[a]) > (cu[b + 1] - cu[b]); });
   int units = 0;
   for (int k = 0; k < n_items; ++k) {
@@ -731,7 +734,7 @@ static eas_status launch_attention_mma(const bf16* qkv, bf16* out, const int32_t
 
 template <bool PT>
 static eas_status launch_attention_tc(const bf16* qkv, bf16* out, const int32_t* cu, int n_items, int H, int hd, int budget,
-                                      cudaStream_t stream, uint32_t* status) {
+                                      cudaStream_t stream, uint32_t* status, bool reverse) {
   AttnTcParams ap{};
   const int d = H * hd;
   const int64_t T = cu[n_items];
@@ -761,7 +764,7 @@ static eas_status launch_attention_tc(const bf16* qkv, bf16* out, const int32_t*
   bool dual = false;
   if (hd == 64 && AttnTcSmem<64, PT>::kDualHeadOk && H >= 2)
     for (int i = 0; i < n_items; ++i) dual = dual || (((cu[i + 1] - cu[i] + kTcTile - 1) / kTcTile) & 1) != 0;
-  attention_schedule(cu, n_items, 2 * kTcTile, H, ap.item_start, ap.item_len, ap.unit_prefix, &ap.total_units, dual);
+  attention_schedule(cu, n_items, 2 * kTcTile, H, ap.item_start, ap.item_len, ap.unit_prefix, &ap.total_units, dual, reverse);
   if (ap.total_units == 0) return EAS_OK;
   const int grid = std::min(budget, ap.total_units);
   static bool attr_set = false;
@@ -780,10 +783,10 @@ static eas_status launch_attention_tc(const bf16* qkv, bf16* out, const int32_t*
 }
 
 static eas_status launch_attention(const bf16* qkv, bf16* out, const int32_t* cu, int n_items, int H, int hd, int budget,
-                                   cudaStream_t stream, int impl, uint32_t* status) {
+                                   cudaStream_t stream, int impl, uint32_t* status, bool reverse = false) {
   if (impl == 1) return launch_attention_mma(qkv, out, cu, n_items, H, hd, budget, stream);
-  if (impl == 2) return launch_attention_tc<false>(qkv, out, cu, n_items, H, hd, budget, stream, status);
-  return launch_attention_tc<true>(qkv, out, cu, n_items, H, hd, budget, stream, status);
+  if (impl == 2) return launch_attention_tc<false>(qkv, out, cu, n_items, H, hd, budget, stream, status, reverse);
+  return launch_attention_tc<true>(qkv, out, cu, n_items, H, hd, budget, stream, status, reverse);
 }
 
 // ------------------------------------------------------------------------------------ the forward pass
@@ -934,10 +937,14 @@ static eas_status encode_impl(eas_encoder* e, const eas_packed_inputs* in, void*
   }
 
   // ---- transformer blocks
+  // Consecutive kernels walk the token rows in alternating directions (`dir`): each starts with the rows its producer
+  // wrote last, which are the ones still in L2.  Every row, tile and attention unit is independent of the order.
+  int dir = 0;
   for (int li = 0; li < c.n_layers; ++li) {
     const Layer& L = e->layers[li];
     {
       NormParams np{x, nbuf, L.n1g, L.n1b, nullptr, static_cast<int>(T), d, c.norm_eps};
+      np.reverse = dir; dir ^= 1;
       EAS_TRY(mark(e, EAS_KC_NORM, stream));
       EAS_TRY(launch_norm(ln_kind, false, np, budget, stream)); ++launches;
     }
@@ -946,20 +953,24 @@ static eas_status encode_impl(eas_encoder* e, const eas_packed_inputs* in, void*
       g.A = nbuf; g.a_run = d; g.a_row_elems = d; g.a_rows = T; g.M = static_cast<int>(T); g.lin = &L.qkv;
       g.out = qkv; g.ldo = 3LL * d;
       if (c.pos == EAS_POS_ROPE_2D) { g.rope_cs = rope; g.rope_stride = T; g.rope_pairs = e->hd / 2; g.rope_ncols = 2 * d; g.head_dim = e->hd; }
+      g.reverse = dir; dir ^= 1;
       EAS_TRY(mark(e, EAS_KC_GEMM_QKV, stream));
       EAS_TRY(launch_gemm(g, budget, stream, status)); ++launches;
     }
     EAS_TRY(mark(e, EAS_KC_ATTENTION, stream));
-    EAS_TRY(launch_attention(qkv, obuf, cu, n, c.n_heads, e->hd, budget, stream, e->attn_impl, status)); ++launches;
+    EAS_TRY(launch_attention(qkv, obuf, cu, n, c.n_heads, e->hd, budget, stream, e->attn_impl, status, dir != 0)); ++launches;
+    dir ^= 1;
     {
       GemmCall g;
       g.A = obuf; g.a_run = d; g.a_row_elems = d; g.a_rows = T; g.M = static_cast<int>(T); g.lin = &L.proj;
       g.out_fp32 = 1; g.out = x; g.ldo = d; g.resid = x;
+      g.reverse = dir; dir ^= 1;
       EAS_TRY(mark(e, EAS_KC_GEMM_PROJ, stream));
       EAS_TRY(launch_gemm(g, budget, stream, status)); ++launches;
     }
     {
       NormParams np{x, nbuf, L.n2g, L.n2b, nullptr, static_cast<int>(T), d, c.norm_eps};
+      np.reverse = dir; dir ^= 1;
       EAS_TRY(mark(e, EAS_KC_NORM, stream));
       EAS_TRY(launch_norm(ln_kind, false, np, budget, stream)); ++launches;
     }
@@ -968,6 +979,7 @@ static eas_status encode_impl(eas_encoder* e, const eas_packed_inputs* in, void*
       g.A = nbuf; g.a_run = d; g.a_row_elems = d; g.a_rows = T; g.M = static_cast<int>(T); g.lin = &L.fc1;
       g.act = c.mlp == EAS_MLP_SWIGLU ? ACT_SWIGLU : ACT_GELU;
       g.out = abuf; g.ldo = c.d_mlp;
+      g.reverse = dir; dir ^= 1;
       EAS_TRY(mark(e, EAS_KC_GEMM_FC1, stream));
       EAS_TRY(launch_gemm(g, budget, stream, status)); ++launches;
     }
@@ -975,6 +987,7 @@ static eas_status encode_impl(eas_encoder* e, const eas_packed_inputs* in, void*
       GemmCall g;
       g.A = abuf; g.a_run = c.d_mlp; g.a_row_elems = c.d_mlp; g.a_rows = T; g.M = static_cast<int>(T); g.lin = &L.fc2;
       g.out_fp32 = 1; g.out = x; g.ldo = d; g.resid = x;
+      g.reverse = dir; dir ^= 1;
       EAS_TRY(mark(e, EAS_KC_GEMM_FC2, stream));
       EAS_TRY(launch_gemm(g, budget, stream, status)); ++launches;
     }

@@ -40,6 +40,7 @@ struct NormParams {
   const int* src_rows;   // optional gather: input row of each output row
   int rows, d;
   float eps;
+  int reverse;           // 1: walk the rows last to first (see the row loop)
 };
 
 // One warp per row, the row held in registers (NV float4 per lane), two-pass statistics in fp32.
@@ -63,11 +64,11 @@ __global__ void __launch_bounds__(512, 1) norm_kernel(const NormParams p) {
   const float inv_d = 1.0f / static_cast<float>(p.d);
   pdl_launch_dependents();
   pdl_wait();
-  // Rows are walked from the LAST to the first: the GEMM that produced x wrote its last row panels most recently, so
-  // those rows are the ones still in L2, and the GEMM that consumes the output starts at row 0, which this order writes
-  // last.  (Each row is independent: the order does not change any value.)
+  // The forward pass alternates the direction in which consecutive kernels walk the token rows: a kernel starts with
+  // the rows its producer wrote last, which are the ones still in L2.  (Rows are independent: the order does not change
+  // any value.)
   for (int rr = blockIdx.x * warps_per_cta + warp; rr < p.rows; rr += gridDim.x * warps_per_cta) {
-    const int row = p.rows - 1 - rr;
+    const int row = p.reverse ? p.rows - 1 - rr : rr;
     const long long src = p.src_rows ? p.src_rows[row] : row;
     const float4* xr = reinterpret_cast<const float4*>(p.x + src * p.d);
     float4 v[NV];

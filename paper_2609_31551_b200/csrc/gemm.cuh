@@ -61,6 +61,7 @@ struct alignas(64) GemmParams {
   int kb_per_tap;         // k-blocks per convolution tap (== k_blocks for a plain GEMM)
   int conv_stride;        // 1 for a plain GEMM; row stride of a convolution otherwise
   int m_blocks, n_blocks; // m_blocks counts 128-row blocks (one CTA per tile) or 256-row blocks (CTA pair)
+  int reverse;            // 1: walk the tiles last to first (start with the rows the producer of A wrote last: L2)
   const bf16* bias;       // [N] (for SWIGLU: interleaved gate/up like the W rows)
   void* out;              // bf16 or fp32 [*, ldo]
   long long ldo;          // leading dimension of out (elements)
@@ -147,7 +148,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_kernel(const __grid_cons
       bool ok = true;
       for (int tile = first_tile; tile < num_tiles && ok; tile += tile_step) {
         int mg, nb;
-        tile_coords(tile, p.m_blocks, p.n_blocks, mg, nb);
+        tile_coords(p.reverse ? num_tiles - 1 - tile : tile, p.m_blocks, p.n_blocks, mg, nb);
         const int mb = mg * CTAS + cta_rank;       // this CTA's 128-row block
         for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
           const int s = it % kStages;
@@ -255,7 +256,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_kernel(const __grid_cons
     };
     for (int tile = first_tile; tile < num_tiles && ok; tile += tile_step, ++tcount) {
       int mg, nb;
-      tile_coords(tile, p.m_blocks, p.n_blocks, mg, nb);
+      tile_coords(p.reverse ? num_tiles - 1 - tile : tile, p.m_blocks, p.n_blocks, mg, nb);
       const int mb = mg * CTAS + cta_rank;
       const uint32_t acc = tcount % kAccBuffers;
       const uint32_t acc_ph = (tcount / kAccBuffers) & 1u;
