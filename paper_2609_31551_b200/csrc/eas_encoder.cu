@@ -274,6 +274,22 @@ static eas_status relayout(bf16* dst, const bf16* src, const bf16* src2, long lo
     if (s_ != EAS_OK) return s_; \
   } while (0)
 
+// Kernel attributes (the dynamic shared-memory limit) belong to a device's context: they are set once per DEVICE, the
+// first time a launch site is reached with that device current.
+struct OncePerDevice {
+  std::mutex m;
+  bool done[64] = {};
+  // true exactly once per device ordinal (false for ordinals past the table: the attribute is then set every time)
+  bool first() {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return true;
+    std::lock_guard<std::mutex> lock(m);
+    if (done[dev]) return false;
+    done[dev] = true;
+    return true;
+  }
+};
+
 static eas_status finish_linear(Linear& L) {
   EAS_TRY(make_w_tmap(&L.tmap, L.w, L.N, L.K, kBN));
   EAS_TRY(make_w_tmap(&L.tmap_half, L.w, L.N, L.K, kBN / 2));
@@ -656,10 +672,9 @@ static eas_status launch_norm_nv(const NormParams& p, int budget, cudaStream_t s
   const int nv = p.d / 128;
 #define EAS_NORM_CASE(NV_)                                                                                         \
   case NV_: {                                                                                                      \
-    static bool attr_set = false;                                                                                  \
-    if (!attr_set) {                                                                                               \
+    static OncePerDevice once;                                                                                     \
+    if (once.first()) {                                                                                            \
       CUDA_TRY(cudaFuncSetAttribute(norm_kernel<NV_, KIND, F32>, cudaFuncAttributeMaxDynamicSharedMemorySize, kOnePerSmSmem)); \
-      attr_set = true;                                                                                             \
     }                                                                                                              \
     EAS_TRY(launch_kernel(norm_kernel<NV_, KIND, F32>, std::min(budget, (p.rows + 15) / 16), 512, kOnePerSmSmem, stream, p)); \
     break;                                                                                                         \
@@ -720,11 +735,10 @@ static eas_status launch_attention_mma(const bf16* qkv, bf16* out, const int32_t
   attention_schedule(cu, n_items, kAttnBQ, H, ap.item_start, ap.item_len, ap.unit_prefix, &ap.total_units);
   if (ap.total_units == 0) return EAS_OK;
   const int grid = std::min(budget, ap.total_units);
-  static bool attr_set = false;
-  if (!attr_set) {
+  static OncePerDevice once;
+  if (once.first()) {
     CUDA_TRY(cudaFuncSetAttribute(attn_mma_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, kOnePerSmSmem));
     CUDA_TRY(cudaFuncSetAttribute(attn_mma_kernel<80>, cudaFuncAttributeMaxDynamicSharedMemorySize, kOnePerSmSmem));
-    attr_set = true;
   }
   static_assert(attn_mma_smem_bytes<80>() <= kOnePerSmSmem, "attention tile does not fit");
   if (hd == 64) return launch_kernel(attn_mma_kernel<64>, grid, kAttnThreads, kOnePerSmSmem, stream, ap);
@@ -767,13 +781,12 @@ static eas_status launch_attention_tc(const bf16* qkv, bf16* out, const int32_t*
   attention_schedule(cu, n_items, 2 * kTcTile, H, ap.item_start, ap.item_len, ap.unit_prefix, &ap.total_units, dual, reverse);
   if (ap.total_units == 0) return EAS_OK;
   const int grid = std::min(budget, ap.total_units);
-  static bool attr_set = false;
-  if (!attr_set) {
+  static OncePerDevice once;
+  if (once.first()) {
     CUDA_TRY(cudaFuncSetAttribute(attn_tc_kernel<64, PT>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttnTcSmem<64, PT>::kBytes));
     CUDA_TRY(cudaFuncSetAttribute(attn_tc_kernel<80, PT>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttnTcSmem<80, PT>::kBytes));
     if (AttnTcSmem<64, PT>::kDualHeadOk)
       CUDA_TRY(cudaFuncSetAttribute(attn_tc_kernel<64, PT, AttnTcSmem<64, PT>::kDualHeadOk>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttnTcSmem<64, PT>::kBytes));
-    attr_set = true;
   }
   if (hd == 64 && dual)
     return launch_kernel(attn_tc_kernel<64, PT, AttnTcSmem<64, PT>::kDualHeadOk>, grid, kTcThreads, AttnTcSmem<64, PT>::kBytes, stream, ap);
@@ -894,8 +907,8 @@ static eas_status encode_impl(eas_encoder* e, const eas_packed_inputs* in, void*
     AudioStageParams sp{};
     sp.data = static_cast<const bf16*>(in->data); sp.mel_pad = mel_pad; sp.h1_pad = h1_pad;
     sp.n_mel = c.in_channels; sp.d_model = d; sp.padded_rows = static_cast<int>(pl.padded_rows); sp.items = items;
-    static bool attr_set = false;
-    if (!attr_set) { CUDA_TRY(cudaFuncSetAttribute(audio_stage_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kOnePerSmSmem)); attr_set = true; }
+    static OncePerDevice once;
+    if (once.first()) CUDA_TRY(cudaFuncSetAttribute(audio_stage_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kOnePerSmSmem));
     EAS_TRY(mark(e, EAS_KC_EMBED_GATHER, stream));
     EAS_TRY(launch_kernel(audio_stage_kernel, budget, 512, kOnePerSmSmem, stream, sp));
     ++launches;
@@ -918,8 +931,8 @@ static eas_status encode_impl(eas_encoder* e, const eas_packed_inputs* in, void*
     ip.channels = c.in_channels; ip.patch = c.patch; ip.tpatch = c.temporal_patch;
     ip.merge_order = c.family == EAS_FAMILY_VIT_ROPE_MERGER ? 1 : 0;
     ip.items = items;
-    static bool attr_set = false;
-    if (!attr_set) { CUDA_TRY(cudaFuncSetAttribute(im2col_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kOnePerSmSmem)); attr_set = true; }
+    static OncePerDevice once;
+    if (once.first()) CUDA_TRY(cudaFuncSetAttribute(im2col_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kOnePerSmSmem));
     EAS_TRY(mark(e, EAS_KC_EMBED_GATHER, stream));
     EAS_TRY(launch_kernel(im2col_kernel, budget, 512, kOnePerSmSmem, stream, ip));
     ++launches;
@@ -1229,8 +1242,8 @@ extern "C" eas_status eas_kernel_gemm(const void* A, const void* W, const void* 
   if (act < 0 || act > 2 || (act == ACT_SWIGLU && out_fp32)) return fail(EAS_ERR_INVALID_ARG, "bad epilogue selection");
   int budget = 0;
   EAS_TRY(resolve_budget(sm_budget, &budget));
-  static bool attrs_done = false;
-  if (!attrs_done) { EAS_TRY(set_kernel_attributes()); attrs_done = true; }
+  static OncePerDevice once;
+  if (once.first()) EAS_TRY(set_kernel_attributes());
   Linear L;
   L.w = static_cast<const bf16*>(W); L.b = static_cast<const bf16*>(bias); L.N = N; L.K = K;
   EAS_TRY(finish_linear(L));
