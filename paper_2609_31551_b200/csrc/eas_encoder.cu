@@ -1277,6 +1277,11 @@ extern "C" eas_status eas_kernel_attention(const void* qkv, void* out, const int
                           static_cast<cudaStream_t>(stream), impl, status_dev);
 }
 
+#ifdef EAS_GEMM_PROFILE
+extern "C" int eas_debug_gemm_stamps(unsigned long long* host_out /* [32*16] */) {
+  return cudaMemcpyFromSymbol(host_out, eas::g_gemm_dbg, sizeof(unsigned long long) * 32 * 16) == cudaSuccess ? 0 : 1;
+}
+#endif
 #ifdef EAS_ATTN_PROFILE
 extern "C" int eas_debug_attn_stamps(unsigned long long* host_out /* [2*64*12] */) {
   return cudaMemcpyFromSymbol(host_out, eas::g_attn_dbg, sizeof(unsigned long long) * 2 * 64 * 12) == cudaSuccess ? 0 : 1;

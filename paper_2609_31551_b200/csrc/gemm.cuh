@@ -78,6 +78,14 @@ struct alignas(64) GemmParams {
   uint32_t* status;       // device status word
 };
 
+#ifdef EAS_GEMM_PROFILE
+// phase timestamps of epilogue warp 0 of CTA 0 (profiling builds only): [tile][k]
+__device__ unsigned long long g_gemm_dbg[32 * 16];
+#define GEMM_STAMP(k) do { if (blockIdx.x == 0 && ew == 0 && lane == 0 && tcount < 32) g_gemm_dbg[tcount * 16 + (k)] = clock64(); } while (0)
+#else
+#define GEMM_STAMP(k) do { } while (0)
+#endif
+
 __device__ __forceinline__ void tile_coords(int tile, int m_blocks, int n_blocks, int& mb, int& nb) {
   const int per_panel = kPanelM * n_blocks;
   const int panel = tile / per_panel;
@@ -249,9 +257,11 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_kernel(const __grid_cons
     bool ok = true;
     auto release_accumulator = [&](uint32_t acc) {   // this warp has read its part of the accumulator
       tc_fence_before_sync();
+      GEMM_STAMP(12);
       __syncwarp();
+      GEMM_STAMP(13);
       if (lane == 0) {
-        if (CTAS == 2) mbar_arrive_cluster(&acc_empty[acc], 0); else mbar_arrive(&acc_empty[acc]);
+        if (CTAS == 2) mbar_arrive_cluster_relaxed(&acc_empty[acc], 0); else mbar_arrive(&acc_empty[acc]);
       }
     };
     for (int tile = first_tile; tile < num_tiles && ok; tile += tile_step, ++tcount) {
@@ -273,9 +283,12 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_kernel(const __grid_cons
           __syncwarp();
           if (lane == 0) mbar_arrive(&bias_bar[acc]);
         }
+        GEMM_STAMP(0);
         if (!mbar_wait(&acc_full[acc], acc_ph, abort_flag)) { ok = false; break; }
+        GEMM_STAMP(1);
         if (!mbar_wait(&bias_bar[acc], acc_ph, abort_flag)) { ok = false; break; }
         tc_fence_after_sync();
+        GEMM_STAMP(2);
         uint8_t* stage = smem + kStagingOff + ew * 4096;
         uint8_t* srow = stage + lane * 128;
         const int sw = lane & 7;
@@ -361,11 +374,13 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_kernel(const __grid_cons
           tmem_ld_32x32(taddr + pr * 64, r0);
           tmem_ld_32x32(taddr + pr * 64 + 32, r1);
           tmem_ld_wait();
+          GEMM_STAMP(3 + pr * 4);
           float v0[32], v1[32];
 #pragma unroll
           for (int i = 0; i < 32; ++i) { v0[i] = __uint_as_float(r0[i]); v1[i] = __uint_as_float(r1[i]); }
           finish_chunk(v0, pr * 2);
           finish_chunk(v1, pr * 2 + 1);
+          GEMM_STAMP(4 + pr * 4);
           const int col0 = nb * kTileN + half * (128 * NW) + pr * 64;
           if (OUT == OUT_F32) {
             // 32 fp32 columns = one 128-byte staging row; two sub-tiles per round
@@ -396,6 +411,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_kernel(const __grid_cons
           } else {
             // 64 bf16 columns = one 128-byte staging row
             staging_free();
+            GEMM_STAMP(5 + pr * 4);
 #pragma unroll
             for (int h2 = 0; h2 < 2; ++h2) {
               float (&v)[32] = h2 ? v1 : v0;
@@ -406,10 +422,12 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_kernel(const __grid_cons
                                pack_bf16x2(v[8 * q + 4], v[8 * q + 5]), pack_bf16x2(v[8 * q + 6], v[8 * q + 7]));
             }
             if (col0 < p.N) store_subtile(col0);
+            GEMM_STAMP(6 + pr * 4);
           }
         }
         }
         release_accumulator(acc);
+        GEMM_STAMP(11);
         continue;
       }
 

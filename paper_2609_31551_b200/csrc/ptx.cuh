@@ -158,6 +158,18 @@ __device__ __forceinline__ void cluster_sync_all() {
   asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
 // arrive on the barrier at the same shared-memory offset in CTA `cta` of the cluster
+// Arrival at a barrier of CTA `cta` of the cluster WITHOUT memory-release semantics, for hand-offs that carry no data
+// through memory (a TMEM buffer whose loads have completed: tcgen05.wait::ld + tcgen05.fence::before_thread_sync order
+// those).  The releasing form below makes the arriving thread wait until its earlier memory operations are performed at
+// cluster scope, which was measured at 3000-3900 cycles per arrival in the GEMM epilogue (a TMA store just issued).
+__device__ __forceinline__ void mbar_arrive_cluster_relaxed(uint64_t* bar, uint32_t cta) {
+  asm volatile(
+      "{\n\t.reg .b32 ra;\n\t"
+      "mapa.shared::cluster.u32 ra, %0, %1;\n\t"
+      "mbarrier.arrive.relaxed.cluster.shared::cluster.b64 _, [ra];\n\t}"
+      ::"r"(smem_u32(bar)), "r"(cta)
+      : "memory");
+}
 __device__ __forceinline__ void mbar_arrive_cluster(uint64_t* bar, uint32_t cta) {
   asm volatile(
       "{\n\t.reg .b32 ra;\n\t"
