@@ -194,6 +194,24 @@ eas_status eas_encoder_enable_timing(eas_encoder* enc, int32_t on);
  * available), or -1 on a CUDA error. */
 int32_t eas_encoder_timing_read(eas_encoder* enc, int32_t capacity, int32_t* kernel_class, float* ms);
 
+/* ---- SM partition (Section 3.4: the encoder gets a share of the SMs, the co-located prefill worker the rest) ----
+ * eas_sm_partition_create splits the current device's SMs into two disjoint sets with the driver's green contexts
+ * and creates one non-blocking stream in each: side 0 holds at least `sm_encode` SMs (the driver rounds up to its
+ * granularity, 8 SMs on this architecture, and keeps SM pairs together so that CTA-pair clusters still launch), side 1
+ * the remaining ones.  Kernels enqueued on a side's stream run only on that side's SMs, whatever their grid size, so an
+ * encoder call given side 0's stream and sm_budget = eas_sm_partition_sm_count(p, 0) cannot be slowed by a neighbour's
+ * kernels occupying its SMs; L2 and HBM stay shared.  Device memory is shared with the rest of the process.
+ * Errors: EAS_ERR_INVALID_ARG (sm_encode <= 0 or nothing left for side 1), EAS_ERR_UNSUPPORTED (driver without
+ * green contexts), EAS_ERR_CUDA.  The handle owns the streams and contexts: destroy it after the work on them is done
+ * (destroy waits for both streams). */
+typedef struct eas_sm_partition eas_sm_partition;
+eas_status eas_sm_partition_create(int32_t sm_encode, eas_sm_partition** out);
+/* Number of SMs of side 0 (encoder) or 1 (neighbour); 0 for any other argument. */
+int32_t eas_sm_partition_sm_count(const eas_sm_partition* p, int32_t side);
+/* The side's stream (a cudaStream_t), owned by the handle. */
+void* eas_sm_partition_stream(const eas_sm_partition* p, int32_t side);
+void eas_sm_partition_destroy(eas_sm_partition* p);
+
 const char* eas_last_error(void);
 
 void eas_encoder_destroy(eas_encoder* enc);

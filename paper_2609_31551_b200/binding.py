@@ -17,6 +17,7 @@ EXPORTED_SYMBOLS = [
     "eas_encoder_create", "eas_encoder_weight_arena_bytes", "eas_encoder_workspace_bytes", "eas_encoder_out_rows",
     "eas_encode_microbatch", "eas_encode_microbatch_static", "eas_encoder_status", "eas_encoder_last_launch_count", "eas_encoder_set_attention_impl",
     "eas_encoder_set_graph_mode", "eas_encoder_graph_stats", "eas_encoder_enable_timing", "eas_encoder_timing_read", "eas_last_error", "eas_encoder_destroy", "eas_kernel_gemm", "eas_kernel_norm", "eas_kernel_attention",
+    "eas_sm_partition_create", "eas_sm_partition_sm_count", "eas_sm_partition_stream", "eas_sm_partition_destroy",
 ]
 
 
@@ -98,6 +99,14 @@ def load_library():
     lib.eas_kernel_attention.restype = C.c_int
     lib.eas_kernel_attention.argtypes = [C.c_void_p, C.c_void_p, C.POINTER(C.c_int32), C.c_int32, C.c_int32, C.c_int32,
                                          C.c_int32, C.c_void_p, C.c_int32, C.c_void_p]
+    lib.eas_sm_partition_create.restype = C.c_int
+    lib.eas_sm_partition_create.argtypes = [C.c_int32, C.POINTER(C.c_void_p)]
+    lib.eas_sm_partition_sm_count.restype = C.c_int32
+    lib.eas_sm_partition_sm_count.argtypes = [C.c_void_p, C.c_int32]
+    lib.eas_sm_partition_stream.restype = C.c_void_p
+    lib.eas_sm_partition_stream.argtypes = [C.c_void_p, C.c_int32]
+    lib.eas_sm_partition_destroy.restype = None
+    lib.eas_sm_partition_destroy.argtypes = [C.c_void_p]
     _lib = lib
     return lib
 
@@ -266,6 +275,36 @@ class Encoder:
 
     def last_launch_count(self) -> int:
         return self.lib.eas_encoder_last_launch_count(self.handle)
+
+
+class SmPartition:
+    """eas_sm_partition: the device's SMs split into side 0 (the encoder, at least `sm_encode` SMs) and side 1 (the
+    neighbour, the rest), one stream on each (Section 3.4).  `stream(side)` is a torch stream object over the
+    library's stream; the handle owns it, so keep this object alive while the streams are in use."""
+
+    def __init__(self, sm_encode: int):
+        self.lib = load_library()
+        h = C.c_void_p()
+        _check(self.lib.eas_sm_partition_create(int(sm_encode), C.byref(h)))
+        self.handle = h
+        self._streams = [torch.cuda.ExternalStream(self.lib.eas_sm_partition_stream(h, s)) for s in (0, 1)]
+
+    def sm_count(self, side: int) -> int:
+        return self.lib.eas_sm_partition_sm_count(self.handle, side)
+
+    def stream(self, side: int):
+        return self._streams[side]
+
+    def close(self):
+        if self.handle is not None:
+            self.lib.eas_sm_partition_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
 
 
 def kernel_gemm(A, W, bias, act=0, out_fp32=False, resid=None, sm_budget=0, stream=None, out=None, status=None):

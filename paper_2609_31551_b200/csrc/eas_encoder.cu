@@ -1224,6 +1224,96 @@ extern "C" eas_status eas_encoder_status(eas_encoder* e, void* stream_v) {
   return EAS_OK;
 }
 
+// ------------------------------------------------------------------------------------ SM partition (Section 3.4)
+// Two green contexts over disjoint sets of SMs, one stream in each.  The driver calls are looked up at run time (the
+// library does not link libcuda).
+namespace {
+template <typename Fn>
+Fn driver_fn(const char* name) {
+  void* p = nullptr;
+  cudaDriverEntryPointQueryResult q;
+  if (cudaGetDriverEntryPoint(name, &p, cudaEnableDefault, &q) != cudaSuccess || q != cudaDriverEntryPointSuccess) return nullptr;
+  return reinterpret_cast<Fn>(p);
+}
+struct GreenApi {
+  CUresult (*device_get)(CUdevice*, int) = nullptr;
+  CUresult (*get_resource)(CUdevice, CUdevResource*, CUdevResourceType) = nullptr;
+  CUresult (*split)(CUdevResource*, unsigned int*, const CUdevResource*, CUdevResource*, unsigned int, unsigned int) = nullptr;
+  CUresult (*gen_desc)(CUdevResourceDesc*, CUdevResource*, unsigned int) = nullptr;
+  CUresult (*ctx_create)(CUgreenCtx*, CUdevResourceDesc, CUdevice, unsigned int) = nullptr;
+  CUresult (*ctx_destroy)(CUgreenCtx) = nullptr;
+  CUresult (*stream_create)(CUstream*, CUgreenCtx, unsigned int, int) = nullptr;
+  bool load() {
+    device_get = driver_fn<decltype(device_get)>("cuDeviceGet");
+    get_resource = driver_fn<decltype(get_resource)>("cuDeviceGetDevResource");
+    split = driver_fn<decltype(split)>("cuDevSmResourceSplitByCount");
+    gen_desc = driver_fn<decltype(gen_desc)>("cuDevResourceGenerateDesc");
+    ctx_create = driver_fn<decltype(ctx_create)>("cuGreenCtxCreate");
+    ctx_destroy = driver_fn<decltype(ctx_destroy)>("cuGreenCtxDestroy");
+    stream_create = driver_fn<decltype(stream_create)>("cuGreenCtxStreamCreate");
+    return device_get && get_resource && split && gen_desc && ctx_create && ctx_destroy && stream_create;
+  }
+};
+}  // namespace
+
+struct eas_sm_partition {
+  GreenApi api;
+  CUgreenCtx ctx[2] = {nullptr, nullptr};
+  CUstream stream[2] = {nullptr, nullptr};
+  int32_t sm_count[2] = {0, 0};
+};
+
+extern "C" void eas_sm_partition_destroy(eas_sm_partition* p) {
+  if (p == nullptr) return;
+  for (int s = 0; s < 2; ++s) {
+    if (p->stream[s] != nullptr) { cudaStreamSynchronize(p->stream[s]); cudaStreamDestroy(p->stream[s]); }
+    if (p->ctx[s] != nullptr) p->api.ctx_destroy(p->ctx[s]);
+  }
+  delete p;
+}
+
+extern "C" eas_status eas_sm_partition_create(int32_t sm_encode, eas_sm_partition** out) {
+  if (out == nullptr) return fail(EAS_ERR_INVALID_ARG, "eas_sm_partition_create: out is NULL");
+  *out = nullptr;
+  if (sm_encode <= 0) return fail(EAS_ERR_INVALID_ARG, "eas_sm_partition_create: sm_encode = %d", sm_encode);
+  int dev = 0;
+  CUDA_TRY(cudaGetDevice(&dev));
+  CUDA_TRY(cudaFree(nullptr));                       // the primary context exists from here on
+  std::unique_ptr<eas_sm_partition, void (*)(eas_sm_partition*)> p(new eas_sm_partition, eas_sm_partition_destroy);
+  if (!p->api.load()) return fail(EAS_ERR_UNSUPPORTED, "this driver has no green contexts");
+  CUdevice cudev;
+  CUdevResource all, part[2];
+  CUresult r = p->api.device_get(&cudev, dev);
+  if (r == CUDA_SUCCESS) r = p->api.get_resource(cudev, &all, CU_DEV_RESOURCE_TYPE_SM);
+  if (r != CUDA_SUCCESS) return fail(EAS_ERR_CUDA, "cuDeviceGetDevResource failed with code %d", static_cast<int>(r));
+  if (sm_encode >= static_cast<int32_t>(all.sm.smCount))
+    return fail(EAS_ERR_INVALID_ARG, "eas_sm_partition_create: sm_encode = %d leaves nothing of %u SMs", sm_encode, all.sm.smCount);
+  unsigned int groups = 1;
+  r = p->api.split(&part[0], &groups, &all, &part[1], 0, static_cast<unsigned int>(sm_encode));
+  if (r != CUDA_SUCCESS || groups != 1)
+    return fail(EAS_ERR_CUDA, "cuDevSmResourceSplitByCount(%d) failed with code %d (%u groups)", sm_encode, static_cast<int>(r), groups);
+  if (part[1].sm.smCount == 0)
+    return fail(EAS_ERR_INVALID_ARG, "eas_sm_partition_create: %d SMs round up to %u and leave none", sm_encode, part[0].sm.smCount);
+  for (int s = 0; s < 2; ++s) {
+    CUdevResourceDesc desc;
+    r = p->api.gen_desc(&desc, &part[s], 1);
+    if (r == CUDA_SUCCESS) r = p->api.ctx_create(&p->ctx[s], desc, cudev, CU_GREEN_CTX_DEFAULT_STREAM);
+    if (r == CUDA_SUCCESS) r = p->api.stream_create(&p->stream[s], p->ctx[s], CU_STREAM_NON_BLOCKING, 0);
+    if (r != CUDA_SUCCESS) return fail(EAS_ERR_CUDA, "creating the green context of side %d failed with code %d", s, static_cast<int>(r));
+    p->sm_count[s] = static_cast<int32_t>(part[s].sm.smCount);
+  }
+  *out = p.release();
+  return EAS_OK;
+}
+
+extern "C" int32_t eas_sm_partition_sm_count(const eas_sm_partition* p, int32_t side) {
+  return (p != nullptr && (side == 0 || side == 1)) ? p->sm_count[side] : 0;
+}
+
+extern "C" void* eas_sm_partition_stream(const eas_sm_partition* p, int32_t side) {
+  return (p != nullptr && (side == 0 || side == 1)) ? static_cast<void*>(p->stream[side]) : nullptr;
+}
+
 // ------------------------------------------------------------------------------------ single-kernel entry points
 static eas_status resolve_budget(int32_t sm_budget, int* budget) {
   int sm_count = 0;

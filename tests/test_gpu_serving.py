@@ -70,3 +70,48 @@ def test_coresidency_measurement_runs_and_reports_sane_numbers():
               "neighbour_tflops_beside_encoder"):
         assert np.isfinite(r[k]) and r[k] > 0
     assert 0.5 < r["inflation"] < 20
+    g = CR.measure("c0", 4, levels=(0.5,), reps=3, neighbour_shape=(2048, 2048, 2048), partition="green")[0]
+    assert g["partition"] == "green" and g["sm_encode"] >= 74 and g["sm_neighbour"] > 0
+    assert np.isfinite(g["inflation"]) and 0.5 < g["inflation"] < 20
+
+
+def test_sm_partition_splits_the_device_and_the_encoder_runs_on_its_side():
+    """Section 3.4: two disjoint SM sets with a stream each.  The encoder on side 0 gives the bits of an ordinary call
+    (the result does not depend on which or how many SMs run it), with a neighbour busy on side 1 meanwhile."""
+    import paper_2609_31551_b200 as P
+    total = torch.cuda.get_device_properties(0).multi_processor_count
+    part = P.SmPartition(44)
+    n0, n1 = part.sm_count(0), part.sm_count(1)
+    assert n0 >= 44 and n1 > 0 and n0 + n1 <= total
+    assert part.sm_count(2) == 0
+    cfg = S.get_config("c0")
+    enc = P.Encoder(cfg, P.weights_to_device(S.make_weights(cfg)))
+    shapes = [(1, 224, 224)] * 3
+    items = S.make_items(cfg, shapes, seed=41)
+    data, offsets = P.pack_items(items)
+    cu = np.concatenate([[0], np.cumsum([S.tokens_per_item(cfg, s) for s in shapes])]).astype(np.int32)
+    ref = enc.encode_microbatch(data, shapes, offsets, cu)
+    enc.status()
+    torch.cuda.synchronize()
+    a = (torch.randn(2048, 2048, device="cuda") * 0.05).bfloat16()
+    bias = torch.zeros(2048, dtype=torch.bfloat16, device="cuda")
+    s0, s1 = part.stream(0), part.stream(1)
+    nb_out = None
+    for _ in range(8):                                     # the neighbour: GEMMs on side 1's SMs
+        nb_out, nb_status = P.kernel_gemm(a, a, bias, sm_budget=n1, stream=s1)
+    with torch.cuda.stream(s0):
+        out = enc.encode_microbatch(data, shapes, offsets, cu, sm_budget=n0, stream=s0)
+        enc.status(s0)
+        # a grid larger than the side still runs there (its CTAs queue for the side's SMs)
+        out_big = enc.encode_microbatch(data, shapes, offsets, cu, sm_budget=total, stream=s0)
+        enc.status(s0)
+    torch.cuda.synchronize()
+    assert torch.equal(out, ref) and torch.equal(out_big, ref)
+    assert int(nb_status[0]) == 0
+    want = (a.double() @ a.double().T)[:4, :4].cpu().numpy()
+    assert np.allclose(nb_out[:4, :4].double().cpu().numpy(), want, rtol=2e-2, atol=2e-2)
+    part.close()
+    with pytest.raises(P.EasError):
+        P.SmPartition(0)
+    with pytest.raises(P.EasError):
+        P.SmPartition(total)
