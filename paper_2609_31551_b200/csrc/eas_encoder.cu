@@ -594,6 +594,7 @@ struct GemmCall {
   const bf16* pos = nullptr;
   const float2* rope_cs = nullptr;
   int reverse = 0;             // walk the tiles last to first
+  int w_const = 1;             // the weights are constant (set at create time): their loads may start before the stream's earlier work ends
   long long rope_stride = 0;   // rows of the [pair][row] table
   int rope_pairs = 0, rope_ncols = 0, head_dim = 0;
 };
@@ -648,6 +649,7 @@ static eas_status launch_gemm(const GemmCall& g, int budget, cudaStream_t stream
   p.k_blocks = deep ? (p.kb_per_tap + 1) / 2 : p.kb_per_tap * g.taps;
   p.conv_stride = g.conv_stride;
   p.reverse = g.reverse;
+  p.w_const = g.w_const;
   p.m_blocks = (g.M + kBM * ctas - 1) / (kBM * ctas);
   p.n_blocks = (L.N + tile_n - 1) / tile_n;
   p.bias = L.b;
@@ -1340,6 +1342,7 @@ extern "C" eas_status eas_kernel_gemm(const void* A, const void* W, const void* 
   GemmCall g;
   g.A = A; g.a_run = K; g.a_row_elems = K; g.a_rows = M; g.M = M; g.lin = &L; g.act = act; g.out_fp32 = out_fp32;
   g.out = out; g.ldo = act == ACT_SWIGLU ? N / 2 : N; g.resid = out_fp32 ? resid : nullptr;
+  g.w_const = 0;             // W is the caller's tensor: work earlier in the stream may have produced it
   return launch_gemm(g, budget, static_cast<cudaStream_t>(stream), status_dev);
 }
 

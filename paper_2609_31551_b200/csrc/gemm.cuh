@@ -75,6 +75,7 @@ struct alignas(64) GemmParams {
   int rope_pairs;         // pairs per head (head_dim / 2)
   int rope_ncols;         // rotate output columns [0, rope_ncols)
   int head_dim;
+  int w_const;            // W is never written by work earlier in the stream: its loads need not wait for that work
   uint32_t* status;       // device status word
 };
 
@@ -82,8 +83,12 @@ struct alignas(64) GemmParams {
 // phase timestamps of epilogue warp 0 of CTA 0 (profiling builds only): [tile][k]
 __device__ unsigned long long g_gemm_dbg[32 * 16];
 #define GEMM_STAMP(k) do { if (blockIdx.x == 0 && ew == 0 && lane == 0 && tcount < 32) g_gemm_dbg[tcount * 16 + (k)] = clock64(); } while (0)
+// one-off timeline of CTA 0 in nanoseconds (row 31 of the same array)
+__device__ __forceinline__ unsigned long long gemm_globaltimer() { unsigned long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); return t; }
+#define GEMM_TL(k) do { if (blockIdx.x == 0) g_gemm_dbg[31 * 16 + (k)] = gemm_globaltimer(); } while (0)
 #else
 #define GEMM_STAMP(k) do { } while (0)
+#define GEMM_TL(k) do { } while (0)
 #endif
 
 __device__ __forceinline__ void tile_coords(int tile, int m_blocks, int n_blocks, int& mb, int& nb) {
@@ -119,6 +124,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_kernel(const __grid_cons
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
+  if (threadIdx.x == 0) GEMM_TL(0);
   const int num_tiles = p.m_blocks * p.n_blocks;
   const int cta_rank = CTAS == 2 ? static_cast<int>(cluster_ctarank()) : 0;
   const int first_tile = blockIdx.x / CTAS;        // both CTAs of a pair walk the same tiles
@@ -142,8 +148,12 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_kernel(const __grid_cons
   if (CTAS == 2) cluster_sync_all();               // the peer's barriers are initialised before anything signals them
   tc_fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
+  if (threadIdx.x == 0) GEMM_TL(1);
   pdl_launch_dependents();   // the next kernel may set itself up while this one runs
-  pdl_wait();                // everything before this kernel in the stream is complete and visible
+  // everything before this kernel in the stream is complete and visible; the W producer of a GEMM on constant
+  // weights goes ahead and fills the ring's W halves meanwhile (the stages complete once A has arrived too)
+  if (!(p.w_const && warp == kProducerBWarp)) pdl_wait();
+  if (threadIdx.x == 0) GEMM_TL(2);
 
   if (warp == 0 || warp == kProducerBWarp) {
     // ------------------------------------------------------------------ producers: warp 0 loads A, the last warp B
@@ -220,6 +230,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_kernel(const __grid_cons
           const int s = it % kStages;
           const uint32_t ph = (it / kStages) & 1u;
           if (!mbar_wait(&full_bar[s], ph, abort_flag)) { ok = false; break; }
+          if (tcount == 0 && kb == 0) GEMM_TL(3);
           tc_fence_after_sync();
           const uint32_t a_addr = smem_u32(smem + s * kStageBytes);
           const uint32_t b_addr = a_addr + kABytes * KD;
@@ -286,6 +297,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_kernel(const __grid_cons
         GEMM_STAMP(0);
         if (!mbar_wait(&acc_full[acc], acc_ph, abort_flag)) { ok = false; break; }
         GEMM_STAMP(1);
+        if (tcount == 0 && ew == 0 && lane == 0) GEMM_TL(4);
         if (!mbar_wait(&bias_bar[acc], acc_ph, abort_flag)) { ok = false; break; }
         tc_fence_after_sync();
         GEMM_STAMP(2);
@@ -428,6 +440,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_kernel(const __grid_cons
         }
         release_accumulator(acc);
         GEMM_STAMP(11);
+        if (tcount == 0 && ew == 0 && lane == 0) GEMM_TL(5);
         continue;
       }
 
@@ -543,6 +556,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_kernel(const __grid_cons
     }
     // bulk stores still reading the staging buffer must finish before the CTA's shared memory is released
     if (p.use_tma_out && lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+    if (ew == 0 && lane == 0) GEMM_TL(6);
   }
 
   tc_fence_before_sync();
@@ -552,6 +566,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_kernel(const __grid_cons
     tc_fence_after_sync();
     if (CTAS == 2) tmem_dealloc_pair(tmem_base, kTmemCols); else tmem_dealloc(tmem_base, kTmemCols);
   }
+  if (threadIdx.x == 0) GEMM_TL(7);
   if (threadIdx.x == 0 && *abort_flag) atomicCAS(p.status, DEV_OK, DEV_ERR_WAIT_TIMEOUT);
 }
 
