@@ -179,3 +179,100 @@ def test_attention_head_dim_80_key_tile_edges(H):
         torch.cuda.synchronize()
         assert int(st2[0]) == 0
         assert torch.equal(out, out2), budget
+
+
+@pytest.mark.parametrize("hd", [64, 80])
+@pytest.mark.parametrize("case", ["rising", "falling", "peaked", "uniform", "tiny_scores"])
+def test_attention_softmax_degenerate_score_patterns(hd, case):
+    """The online softmax across key tiles under score patterns that stress it: scores that rise with the key index
+    (the running maximum grows in every tile, every earlier partial sum is rescaled), scores that fall (the first
+    tile holds the maximum, later tiles underflow), one dominant key per query with score gaps of hundreds (the
+    output is that key's value row), equal keys (the output is the mean of the values: a closed form), and scores
+    of magnitude 1e-3."""
+    import paper_2609_31551_b200 as P
+    H, lens = 2, [700, 130]
+    T, d = sum(lens), H * hd
+    rng = np.random.Generator(np.random.PCG64(77 + hd))
+    q = _bf16_exact(rng, (T, d))
+    k = _bf16_exact(rng, (T, d))
+    v = _bf16_exact(rng, (T, d))
+    pos = np.concatenate([np.arange(n) for n in lens]).astype(np.float32)[:, None]
+    if case in ("rising", "falling"):
+        # q = all ones, k = +-(index / 64) on every coordinate: score = +-index * hd / 64 / sqrt(hd), a ramp of
+        # 0 ... 87 (hd 64) or 98 (hd 80) over 700 keys
+        q[:] = 1.0
+        k[:] = (pos / 64.0) * (1.0 if case == "rising" else -1.0)
+    elif case == "peaked":
+        q *= 6.0
+        k *= 6.0
+    elif case == "uniform":
+        k[:] = k[0:1]
+    else:
+        q *= 2.0 ** -5
+        k *= 2.0 ** -5
+    qkv = S.round_to_bf16(np.concatenate([q, k, v], axis=1))
+    cu = np.concatenate([[0], np.cumsum(lens)]).astype(np.int32)
+    t = O._t(qkv)
+    ref = torch.cat([O.attention_one_item(t[a:b, :d].reshape(-1, H, hd), t[a:b, d:2 * d].reshape(-1, H, hd),
+                                          t[a:b, 2 * d:].reshape(-1, H, hd)) for a, b in zip(cu[:-1], cu[1:])])
+    if case == "uniform":
+        vv = torch.from_numpy(qkv[:, 2 * d:].astype(np.float64))
+        want = torch.cat([vv[a:b].mean(0, keepdim=True).expand(b - a, -1) for a, b in zip(cu[:-1], cu[1:])])
+        assert (ref - want).abs().max() < 1e-12                      # the oracle against the closed form
+    for impl in (0, 1, 2):
+        out, status = P.kernel_attention(_dev(qkv), cu, H, hd, impl=impl)
+        torch.cuda.synchronize()
+        assert int(status[0]) == 0
+        got = out.double().cpu()
+        assert torch.isfinite(got).all()
+        err = (got - ref).abs().max()
+        assert err <= 2e-2, (case, impl, float(err))
+
+
+@pytest.mark.parametrize("act", [1, 2])
+def test_gemm_activation_over_a_wide_input_range(act):
+    """GELU (erf form) and SwiGLU on pre-activations from -50 to 50: the far tails (exactly x, exactly -0 / 0), the
+    region around zero, and the transition in between, against the oracle's definition.  A has one non-zero per row,
+    so the pre-activation of row i is exactly ramp[i] * W[:, i % K] + b."""
+    import paper_2609_31551_b200 as P
+    M, N, K = 1024, 256, 64
+    A = np.zeros((M, K), np.float32)
+    ramp = S.round_to_bf16(np.linspace(-50.0, 50.0, M).astype(np.float32))
+    A[np.arange(M), np.arange(M) % K] = ramp
+    rng = np.random.Generator(np.random.PCG64(act))
+    W = S.round_to_bf16(np.where(rng.random((N, K)) < 0.5, 1.0, 0.5).astype(np.float32))
+    b = _bf16_exact(rng, (N,), 0.25)
+    y = O.linear(O._t(A), O._t(W), O._t(b))
+    y = O.gelu(y) if act == 1 else O.silu(y[:, 0::2]) * y[:, 1::2]
+    out, status = P.kernel_gemm(_dev(A), _dev(W), _dev(b), act=act)
+    torch.cuda.synchronize()
+    assert int(status[0]) == 0
+    got = out.double().cpu()
+    assert torch.isfinite(got).all()
+    tol = 2.0 ** -8 * y.abs() + 1e-4
+    bad = (got - y).abs() > tol
+    assert not bad.any(), f"{int(bad.sum())} wrong, max err {(got - y).abs().max():.3e}, first {bad.nonzero()[:4].tolist()}"
+
+
+@pytest.mark.parametrize("kind", [0, 1])
+def test_norm_rows_with_large_offsets_and_constant_rows(kind):
+    """LayerNorm / RMSNorm on rows whose mean is a thousand times their spread (a one-pass variance would cancel), on
+    constant rows (variance 0: the result is beta, or gamma * x / sqrt(x^2 + eps)) and on an all-zero row."""
+    import paper_2609_31551_b200 as P
+    d, rows, eps = 1024, 96, 1e-6
+    rng = np.random.Generator(np.random.PCG64(300 + kind))
+    x = rng.standard_normal((rows, d)).astype(np.float32)
+    x[:32] += 1000.0
+    x[32:64] = np.linspace(-3, 3, 32, dtype=np.float32)[:, None]
+    x[64] = 0.0
+    g, b = _bf16_exact(rng, (d,)), _bf16_exact(rng, (d,))
+    ref = O.layer_norm(O._t(x), O._t(g), O._t(b), eps) if kind == 0 else O.rms_norm(O._t(x), O._t(g), eps)
+    y = P.kernel_norm(torch.from_numpy(x).cuda(), _dev(g), _dev(b), kind, eps, out_fp32=True)
+    torch.cuda.synchronize()
+    got = y.double().cpu()
+    assert torch.isfinite(got).all()
+    if kind == 0:
+        # constant rows: beta, up to the rounding of the fp32 mean (one ulp of x, magnified by 1 / sqrt(eps) = 1000)
+        assert (got[32:65] - O._t(b).expand(33, -1)).abs().max() <= 2e-3
+    # fp32 statistics: the mean of a row around 1000 carries 1000 * 2^-24 = 6e-5 of error against a spread of 1
+    assert (got - ref).abs().max() <= 5e-4 * max(1.0, float(ref.abs().max()))
