@@ -339,7 +339,7 @@ def run_cuda(args):
                          "peak_kind": f"sustained bf16, {peaks['source']}",
                          # DRAM bytes of one fc1 launch of this workload from an ncu capture (profiles/gemm_fc1_c1_mb32.md):
                          # 46.4 MB read + 97.8 MB written against 197.5 MB algorithmic (part of the output still in L2)
-                         "traffic": 144.2e6 if (args.config == "c1" and args.micro_batch == 32) else None,
+                         "traffic": 143.6e6 if (args.config == "c1" and args.micro_batch == 32) else None,
                          "traffic_note": "dram read+write bytes of one fc1 GEMM launch (ncu); algorithmic 197.5e6",
                          "launches_per_step": gemm_launch, "avg_launch_ms": gemm_ms / max(gemm_launch, 1)},
             "roofline_other": other_rooflines(cfg, shapes, f, acc, n_prof, peaks),
