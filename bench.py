@@ -205,6 +205,8 @@ def run_cuda(args):
     f = flops_of(cfg, shapes)
     T = f["tokens"]
     budget = args.sm_budget
+    if args.split_k:
+        enc.set_split_k(True)          # before any workspace is sized
     if args.graph:
         # the launch-overhead path: captured forward passes need a stream of their own
         torch.cuda.set_stream(torch.cuda.Stream())
@@ -324,7 +326,7 @@ def run_cuda(args):
                        "tokens_per_step": T, "sm_budget": budget if budget else "all",
                        "l2": "working set (weights + activations) larger than L2; no flush",
                        "parallelism": "replicas" if world > 1 else "single",
-                       "launch": "cuda graph replay" if args.graph else "one launch per kernel"},
+                       "launch": ("cuda graph replay" if args.graph else "one launch per kernel") + (", split K" if args.split_k else "")},
             "items_per_sec": total_items * args.steps / (ms * 1e-3),
             "tflops": total_flops / (step_ms * 1e-3) / 1e12,
             "frac_of_bf16_peak": {"burst_measured": f["total"] / (step_ms * 1e-3) / 1e12 / peaks["burst"],
@@ -380,6 +382,8 @@ def main():
     ap.add_argument("--micro-batch", type=int, default=32)
     ap.add_argument("--sm-budget", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--split-k", action="store_true",
+                    help="split the K loop of the residual GEMMs when a micro-batch has fewer tiles than SMs (latency path)")
     ap.add_argument("--graph", action="store_true",
                     help="replay captured forward passes (CUDA graphs): the launch-overhead path for small micro-batches")
     args = ap.parse_args()

@@ -168,6 +168,18 @@ int32_t eas_encoder_last_launch_count(const eas_encoder* enc);
  * testing. */
 eas_status eas_encoder_set_attention_impl(eas_encoder* enc, int32_t impl);
 
+/* Split K for small micro-batches (default off; part of the latency path, like the graph mode below).  With few tokens
+ * the residual GEMMs of a block (x += o W_proj^T, x += h W_fc2^T) have fewer tiles than the device has SMs, and the K
+ * loop of one tile is the whole kernel.  With on = 1, when tiles x s <= SMs and K / s >= 1024 (s = 4 or 2; a function of
+ * the token count, the layer sizes and the device, never of sm_budget), s CTAs share a tile's K range: the first adds its
+ * sum and the bias into the residual stream as usual, the others store bare partial sums, and the normalisation kernel
+ * that follows adds those to the row in a fixed order before normalising it.  Results stay deterministic and independent
+ * of sm_budget, but no longer of what else is in the micro-batch: an item encoded alone (split) and the same item in a
+ * large micro-batch (not split) differ in the last bits, which is why the mode is off unless asked for (off: every
+ * item's embeddings are bit-identical whatever it is packed with).  eas_encoder_workspace_bytes follows the mode (the
+ * partial sums need scratch): set it before sizing the workspace. */
+eas_status eas_encoder_set_split_k(eas_encoder* enc, int32_t on);
+
 /* Launch-overhead path for small micro-batches (Section 3.2: a forward pass at small batch size is dominated by
  * kernel-launch and scheduling overhead).  mode 1: eas_encode_microbatch / _static capture the launches of a
  * micro-batch into a CUDA graph the first time they see it and replay the graph afterwards (one driver call per

@@ -151,6 +151,7 @@ struct eas_encoder {
   const bf16 *cls = nullptr, *pos = nullptr, *eng = nullptr, *enb = nullptr, *fng = nullptr, *fnb = nullptr, *hng = nullptr;
   std::vector<Layer> layers;
   int attn_impl = 0;
+  int split_k = 0;            // small micro-batches split the K loop of the residual GEMMs (eas_encoder_set_split_k)
   int last_launches = 0;
   uint32_t* last_status = nullptr;
   // optional per-kernel timing: one event before every launch and one after the last
@@ -300,7 +301,13 @@ static eas_status finish_linear(Linear& L) {
 typedef void (*GemmKernel)(GemmParams);
 // ctas: 1 = one CTA per 128x256 tile; 2 = CTA pair per 256x256 tile; 3 = CTA pair per 256x512 tile ("wide");
 // deep (pair tiles only): two 64-wide k-blocks per stage and TMA operation
-static GemmKernel gemm_kernel_for(int act, int out_fp32, int ctas, bool deep = false) {
+static GemmKernel gemm_kernel_for(int act, int out_fp32, int ctas, bool deep = false, bool split = false) {
+  if (split) {             // split K: the fp32 residual GEMMs only
+    if (act != ACT_NONE || !out_fp32) return nullptr;
+    if (ctas == 3) return gemm_kernel<ACT_NONE, OUT_F32, 2, 2, 1, true>;
+    if (ctas == 2) return deep ? gemm_kernel<ACT_NONE, OUT_F32, 2, 1, 2, true> : gemm_kernel<ACT_NONE, OUT_F32, 2, 1, 1, true>;
+    return gemm_kernel<ACT_NONE, OUT_F32, 1, 1, 1, true>;
+  }
   if (ctas == 3) {
     if (act == ACT_NONE && !out_fp32) return gemm_kernel<ACT_NONE, OUT_BF16, 2, 2>;
     if (act == ACT_GELU && !out_fp32) return gemm_kernel<ACT_GELU, OUT_BF16, 2, 2>;
@@ -331,6 +338,8 @@ static eas_status set_kernel_attributes() {
     for (int ctas = 1; ctas <= 3; ++ctas)
       for (int act = 0; act < 3; ++act)
         for (int f32 = 0; f32 < 2; ++f32) {
+          GemmKernel ks = gemm_kernel_for(act, f32, ctas, deep != 0, true);
+          if (ks != nullptr) CUDA_TRY(cudaFuncSetAttribute(ks, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmemBytes));
           GemmKernel k = gemm_kernel_for(act, f32, ctas, deep != 0);
           if (k != nullptr)
             CUDA_TRY(cudaFuncSetAttribute(reinterpret_cast<const void*>(k), cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmemBytes));
@@ -487,15 +496,34 @@ extern "C" eas_status eas_encoder_set_attention_impl(eas_encoder* enc, int32_t i
   return EAS_OK;
 }
 
+extern "C" eas_status eas_encoder_set_split_k(eas_encoder* enc, int32_t on) {
+  if (enc == nullptr) return fail(EAS_ERR_INVALID_ARG, "encoder is null");
+  enc->split_k = on != 0 ? 1 : 0;
+  return EAS_OK;
+}
+
 extern "C" int32_t eas_encoder_last_launch_count(const eas_encoder* enc) { return enc ? enc->last_launches : 0; }
 
 // ------------------------------------------------------------------------------------ workspace plan
 namespace {
 struct Plan {
-  size_t status, x, n, qkv, o, a, embed_a, row_map, pos_idx, head_src, rope, mel_pad, h1_pad, conv1_map, total;
+  size_t status, x, n, qkv, o, a, embed_a, row_map, pos_idx, head_src, rope, mel_pad, h1_pad, conv1_map, part, total;
+  int splits_proj, splits_fc2;     // split-K factors of the two residual GEMMs of a block (1: off)
+  int64_t part_rows;               // rows of one split's region of the partial-sum scratch
   int64_t T, embed_rows, padded_rows, out_rows;
 };
 }  // namespace
+
+// Split-K factor of a residual GEMM x[M, N] += A[M, K] W^T with few tiles (small micro-batches: the K loop of one tile is
+// the whole kernel, and most SMs have no tile).  A function of the shape and the device only, never of the SM budget, so
+// that results do not depend on the budget; every split is a whole number of 128-wide k-steps, so that they do not
+// depend on the tile shape either.
+static int pick_splits(int64_t M, int64_t N, int64_t K, int sm_count) {
+  const int64_t items = ((M + kBM - 1) / kBM) * ((N + kBN - 1) / kBN);
+  for (int s = 4; s >= 2; s >>= 1)
+    if (items * s <= sm_count && K % (s * 2 * kBK) == 0 && K / s >= 1024) return s;
+  return 1;
+}
 
 static Plan make_plan(const eas_encoder* e, int64_t T, int n_items) {
   const eas_arch_config& c = e->cfg;
@@ -523,6 +551,10 @@ static Plan make_plan(const eas_encoder* e, int64_t T, int n_items) {
   p.mel_pad = take(static_cast<size_t>(p.padded_rows) * c.in_channels * 2);
   p.h1_pad = take(static_cast<size_t>(p.padded_rows) * d * 2);
   p.conv1_map = take(static_cast<size_t>(p.padded_rows) * 4);
+  p.splits_proj = e->split_k ? pick_splits(T, c.d_model, c.d_model, e->sm_count) : 1;
+  p.splits_fc2 = e->split_k ? pick_splits(T, c.d_model, c.d_mlp, e->sm_count) : 1;
+  p.part_rows = (T + 2 * kBM - 1) / (2 * kBM) * (2 * kBM);
+  p.part = take(static_cast<size_t>(std::max(p.splits_proj, p.splits_fc2) - 1) * p.part_rows * d * 4);
   p.total = off;
   return p;
 }
@@ -595,6 +627,9 @@ struct GemmCall {
   const float2* rope_cs = nullptr;
   int reverse = 0;             // walk the tiles last to first
   int w_const = 1;             // the weights are constant (set at create time): their loads may start before the stream's earlier work ends
+  int splits = 1;              // split K (see GemmParams::splits); the partial sums of splits 1.. go to `part`
+  float* part = nullptr;       // [(splits - 1) * part_rows, N] fp32
+  int64_t part_rows = 0;
   long long rope_stride = 0;   // rows of the [pair][row] table
   int rope_pairs = 0, rope_ncols = 0, head_dim = 0;
 };
@@ -622,12 +657,12 @@ static eas_status launch_gemm(const GemmCall& g, int budget, cudaStream_t stream
   if (budget >= 2) {
     const long long pairs = budget / 2;
     const long long m128 = (g.M + kBM - 1) / kBM, m256 = (g.M + 2 * kBM - 1) / (2 * kBM);
-    const double cost_single = waves(m128 * n256, budget) * kb * 0.47;
-    const double cost_pair = waves(m256 * n256, pairs) * kb * (g.conv_stride == 1 && g.taps == 1 ? 0.40 : 0.43);
+    const double cost_single = waves(m128 * n256 * g.splits, budget) * kb / g.splits * 0.47;
+    const double cost_pair = waves(m256 * n256 * g.splits, pairs) * kb / g.splits * (g.conv_stride == 1 && g.taps == 1 ? 0.40 : 0.43);
     ctas = cost_single < cost_pair ? 1 : 2;
     // wide tiles: long reductions whose output splits evenly into 512-column blocks, plain TMA-stored epilogue
     if (tma_out && g.act != ACT_SWIGLU && k_total >= 2048 && L.N % 512 == 0 && gemm_kernel_for(g.act, g.out_fp32, 3) != nullptr) {
-      const double cost_wide = waves(m256 * (L.N / (2 * kBN)), pairs) * (kb * 0.75 + 4.0);
+      const double cost_wide = waves(m256 * (L.N / (2 * kBN)) * g.splits, pairs) * (kb / g.splits * 0.75 + 4.0);
       if (cost_wide < std::min(cost_single, cost_pair)) { ctas = 2; wide = true; }
     }
 #ifdef EAS_GEMM_FORCE_TILE   // calibration builds only: 1 single CTA, 2 pair, 3 wide pair (where a wide kernel exists)
@@ -650,6 +685,17 @@ static eas_status launch_gemm(const GemmCall& g, int budget, cudaStream_t stream
   p.conv_stride = g.conv_stride;
   p.reverse = g.reverse;
   p.w_const = g.w_const;
+  p.splits = 1;
+  p.kb_per_split = p.k_blocks;
+  if (g.splits > 1) {
+    if (!tma_out || !g.out_fp32 || g.resid != g.out || g.taps != 1 || g.conv_stride != 1 || g.part == nullptr ||
+        g.a_run % (g.splits * 2 * kBK) != 0 || g.part_rows % (2 * kBM) != 0 || g.part_rows < g.M)
+      return fail(EAS_ERR_UNSUPPORTED, "split K needs an in-place fp32 residual GEMM whose K is a multiple of %d", g.splits * 2 * kBK);
+    p.splits = g.splits;
+    p.kb_per_split = p.k_blocks / g.splits;
+    p.part_rows = static_cast<int>(g.part_rows);
+    EAS_TRY(make_out_tmap(&p.tma_part, g.part, true, L.N, L.N, static_cast<int64_t>(g.splits - 1) * g.part_rows));
+  }
   p.m_blocks = (g.M + kBM * ctas - 1) / (kBM * ctas);
   p.n_blocks = (L.N + tile_n - 1) / tile_n;
   p.bias = L.b;
@@ -663,22 +709,22 @@ static eas_status launch_gemm(const GemmCall& g, int budget, cudaStream_t stream
     const int64_t out_cols = g.act == ACT_SWIGLU ? L.N / 2 : L.N;
     EAS_TRY(make_out_tmap(&p.tma_out, g.out, g.out_fp32 != 0, out_cols, g.ldo, g.M));
   }
-  const int tiles = p.m_blocks * p.n_blocks;
-  GemmKernel kern = gemm_kernel_for(g.act, g.out_fp32, wide ? 3 : ctas, deep);
+  const int tiles = p.m_blocks * p.n_blocks * p.splits;
+  GemmKernel kern = gemm_kernel_for(g.act, g.out_fp32, wide ? 3 : ctas, deep, p.splits > 1);
   if (kern == nullptr) return fail(EAS_ERR_UNSUPPORTED, "no GEMM epilogue for act=%d out_fp32=%d", g.act, g.out_fp32);
   return launch_kernel(kern, std::min(budget / ctas, tiles) * ctas, kGemmThreads, kGemmSmemBytes, stream, p, ctas);
 }
 
-template <int KIND, bool F32>
+template <int KIND, bool F32, bool PART = false>
 static eas_status launch_norm_nv(const NormParams& p, int budget, cudaStream_t stream) {
   const int nv = p.d / 128;
 #define EAS_NORM_CASE(NV_)                                                                                         \
   case NV_: {                                                                                                      \
     static OncePerDevice once;                                                                                     \
     if (once.first()) {                                                                                            \
-      CUDA_TRY(cudaFuncSetAttribute(norm_kernel<NV_, KIND, F32>, cudaFuncAttributeMaxDynamicSharedMemorySize, kOnePerSmSmem)); \
+      CUDA_TRY(cudaFuncSetAttribute(norm_kernel<NV_, KIND, F32, PART>, cudaFuncAttributeMaxDynamicSharedMemorySize, kOnePerSmSmem)); \
     }                                                                                                              \
-    EAS_TRY(launch_kernel(norm_kernel<NV_, KIND, F32>, std::min(budget, (p.rows + 15) / 16), 512, kOnePerSmSmem, stream, p)); \
+    EAS_TRY(launch_kernel(norm_kernel<NV_, KIND, F32, PART>, std::min(budget, (p.rows + 15) / 16), 512, kOnePerSmSmem, stream, p)); \
     break;                                                                                                         \
   }
   switch (nv) {
@@ -695,6 +741,11 @@ static eas_status launch_norm_nv(const NormParams& p, int budget, cudaStream_t s
 static eas_status launch_norm(int kind, bool out_fp32, const NormParams& p, int budget, cudaStream_t stream) {
   if (p.rows <= 0) return EAS_OK;
   if (p.d % 128 != 0 || p.d > 2048) return fail(EAS_ERR_UNSUPPORTED, "norm width %d (need a multiple of 128, at most 2048)", p.d);
+  if (p.n_part > 0) {        // split-K partial sums to add first: the residual blocks' bf16 normalisations only
+    if (out_fp32 || p.src_rows != nullptr || p.x_rw == nullptr || p.part == nullptr || kind == NORM_CAST)
+      return fail(EAS_ERR_UNSUPPORTED, "partial sums are added by LayerNorm / RMSNorm with bf16 output only");
+    return kind == NORM_LN ? launch_norm_nv<NORM_LN, false, true>(p, budget, stream) : launch_norm_nv<NORM_RMS, false, true>(p, budget, stream);
+  }
   if (kind == NORM_LN) return out_fp32 ? launch_norm_nv<NORM_LN, true>(p, budget, stream) : launch_norm_nv<NORM_LN, false>(p, budget, stream);
   if (kind == NORM_RMS) return out_fp32 ? launch_norm_nv<NORM_RMS, true>(p, budget, stream) : launch_norm_nv<NORM_RMS, false>(p, budget, stream);
   if (kind == NORM_CAST) return out_fp32 ? fail(EAS_ERR_UNSUPPORTED, "fp32 cast") : launch_norm_nv<NORM_CAST, false>(p, budget, stream);
@@ -879,6 +930,8 @@ static eas_status encode_impl(eas_encoder* e, const eas_packed_inputs* in, void*
   bf16* mel_pad = reinterpret_cast<bf16*>(ws + pl.mel_pad);
   bf16* h1_pad = reinterpret_cast<bf16*>(ws + pl.h1_pad);
   int* conv1_map = reinterpret_cast<int*>(ws + pl.conv1_map);
+  float* part = reinterpret_cast<float*>(ws + pl.part);
+  int pending_parts = 0;      // split-K partial sums of the last residual GEMM, to be added by the next normalisation
   int launches = 0;
   e->last_status = status;
 
@@ -959,6 +1012,7 @@ static eas_status encode_impl(eas_encoder* e, const eas_packed_inputs* in, void*
     const Layer& L = e->layers[li];
     {
       NormParams np{x, nbuf, L.n1g, L.n1b, nullptr, static_cast<int>(T), d, c.norm_eps};
+      np.part = part; np.part_stride = pl.part_rows * d; np.n_part = pending_parts; np.x_rw = x; pending_parts = 0;
       np.reverse = dir; dir ^= 1;
       EAS_TRY(mark(e, EAS_KC_NORM, stream));
       EAS_TRY(launch_norm(ln_kind, false, np, budget, stream)); ++launches;
@@ -979,12 +1033,14 @@ static eas_status encode_impl(eas_encoder* e, const eas_packed_inputs* in, void*
       GemmCall g;
       g.A = obuf; g.a_run = d; g.a_row_elems = d; g.a_rows = T; g.M = static_cast<int>(T); g.lin = &L.proj;
       g.out_fp32 = 1; g.out = x; g.ldo = d; g.resid = x;
+      g.splits = pl.splits_proj; g.part = part; g.part_rows = pl.part_rows; pending_parts = g.splits - 1;   // norm2 follows
       g.reverse = dir; dir ^= 1;
       EAS_TRY(mark(e, EAS_KC_GEMM_PROJ, stream));
       EAS_TRY(launch_gemm(g, budget, stream, status)); ++launches;
     }
     {
       NormParams np{x, nbuf, L.n2g, L.n2b, nullptr, static_cast<int>(T), d, c.norm_eps};
+      np.part = part; np.part_stride = pl.part_rows * d; np.n_part = pending_parts; np.x_rw = x; pending_parts = 0;
       np.reverse = dir; dir ^= 1;
       EAS_TRY(mark(e, EAS_KC_NORM, stream));
       EAS_TRY(launch_norm(ln_kind, false, np, budget, stream)); ++launches;
@@ -1002,6 +1058,9 @@ static eas_status encode_impl(eas_encoder* e, const eas_packed_inputs* in, void*
       GemmCall g;
       g.A = abuf; g.a_run = c.d_mlp; g.a_row_elems = c.d_mlp; g.a_rows = T; g.M = static_cast<int>(T); g.lin = &L.fc2;
       g.out_fp32 = 1; g.out = x; g.ldo = d; g.resid = x;
+      if (li + 1 < c.n_layers) {      // the next block's first normalisation adds the partial sums
+        g.splits = pl.splits_fc2; g.part = part; g.part_rows = pl.part_rows; pending_parts = g.splits - 1;
+      }
       g.reverse = dir; dir ^= 1;
       EAS_TRY(mark(e, EAS_KC_GEMM_FC2, stream));
       EAS_TRY(launch_gemm(g, budget, stream, status)); ++launches;
@@ -1062,7 +1121,7 @@ static eas_status encode_cached(eas_encoder* e, const eas_packed_inputs* in, voi
   const int n = in->n_items;
   std::vector<int64_t> key;
   key.reserve(8 + 5 * static_cast<size_t>(n) + 1);
-  key.push_back(n); key.push_back(sm_budget); key.push_back(e->attn_impl);
+  key.push_back(n); key.push_back(sm_budget); key.push_back(e->attn_impl * 2 + e->split_k);
   key.push_back(static_cast<int64_t>(reinterpret_cast<uintptr_t>(in->data)));
   key.push_back(static_cast<int64_t>(reinterpret_cast<uintptr_t>(workspace)));
   key.push_back(static_cast<int64_t>(workspace_bytes));

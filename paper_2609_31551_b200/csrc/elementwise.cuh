@@ -41,10 +41,17 @@ struct NormParams {
   int rows, d;
   float eps;
   int reverse;           // 1: walk the rows last to first (see the row loop)
+  // Split-K partial sums of the GEMM that produced x (see GemmParams::splits): n_part matrices [part_rows, d], added to
+  // the row in index order before anything else; the completed row is written back to x_rw (== x).
+  const float* part;
+  long long part_stride; // elements between consecutive partial matrices
+  int n_part;
+  float* x_rw;
 };
 
 // One warp per row, the row held in registers (NV float4 per lane), two-pass statistics in fp32.
-template <int NV, int KIND, bool OUT_FP32>
+// PART: the launch adds split-K partial sums to the rows first (a kernel of its own: the ordinary one stays as lean as it was).
+template <int NV, int KIND, bool OUT_FP32, bool PART = false>
 __global__ void __launch_bounds__(512, 1) norm_kernel(const NormParams p) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int warps_per_cta = blockDim.x >> 5;
@@ -74,6 +81,19 @@ __global__ void __launch_bounds__(512, 1) norm_kernel(const NormParams p) {
     float4 v[NV];
 #pragma unroll
     for (int i = 0; i < NV; ++i) v[i] = xr[i * 32 + lane];
+    if (PART) {
+      for (int s = 0; s < p.n_part; ++s) {
+        const float4* pr = reinterpret_cast<const float4*>(p.part + s * p.part_stride + src * p.d);
+#pragma unroll
+        for (int i = 0; i < NV; ++i) {
+          const float4 t = pr[i * 32 + lane];
+          v[i].x += t.x; v[i].y += t.y; v[i].z += t.z; v[i].w += t.w;
+        }
+      }
+      float4* xw = reinterpret_cast<float4*>(p.x_rw + src * p.d);
+#pragma unroll
+      for (int i = 0; i < NV; ++i) xw[i * 32 + lane] = v[i];
+    }
     float mean = 0.f, rstd = 1.f;
     if (KIND == NORM_LN) {
       float s = 0.f;

@@ -76,6 +76,14 @@ struct alignas(64) GemmParams {
   int rope_ncols;         // rotate output columns [0, rope_ncols)
   int head_dim;
   int w_const;            // W is never written by work earlier in the stream: its loads need not wait for that work
+  // Split K (fp32 residual GEMMs with few tiles): a work item is (tile, split); split s accumulates k-blocks
+  // [s * kb_per_split, (s + 1) * kb_per_split).  Split 0 runs the ordinary epilogue (bias, reduce-add into the residual
+  // stream); split s > 0 stores its bare partial sums into rows [(s - 1) * part_rows, ...) of the fp32 scratch matrix
+  // behind tma_part, and the normalisation kernel that follows adds them to the residual rows in a fixed order.
+  int splits;             // >= 1
+  int kb_per_split;
+  int part_rows;          // rows of one split's region of the scratch matrix (a multiple of the tile height)
+  CUtensorMap tma_part;   // [(splits - 1) * part_rows, N] fp32, 32-row boxes of 32 columns
   uint32_t* status;       // device status word
 };
 
@@ -100,7 +108,8 @@ __device__ __forceinline__ void tile_coords(int tile, int m_blocks, int n_blocks
   mb = panel * kPanelM + (within - nb * rows_here);
 }
 
-template <int ACT, int OUT, int CTAS, int NW, int KD = 1>
+// SPLIT: the launch splits K (GemmParams::splits > 1); the ordinary instantiations keep their code free of it.
+template <int ACT, int OUT, int CTAS, int NW, int KD = 1, bool SPLIT = false>
 __global__ void __launch_bounds__(kGemmThreads, 1) gemm_kernel(const __grid_constant__ GemmParams p) {
   static_assert(NW == 1 || (CTAS == 2 && ACT != ACT_SWIGLU), "wide tiles: CTA pairs, no gated epilogue");
   static_assert(KD == 1 || KD == 2, "one or two 64-wide k-blocks per stage");
@@ -126,6 +135,9 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_kernel(const __grid_cons
   const int lane = threadIdx.x & 31;
   if (threadIdx.x == 0) GEMM_TL(0);
   const int num_tiles = p.m_blocks * p.n_blocks;
+  const int n_splits = SPLIT ? p.splits : 1;
+  const int kb_per_split = SPLIT ? p.kb_per_split : p.k_blocks;
+  const int num_work = num_tiles * n_splits;       // work items: (tile, split), the splits of a tile on neighbouring CTAs
   const int cta_rank = CTAS == 2 ? static_cast<int>(cluster_ctarank()) : 0;
   const int first_tile = blockIdx.x / CTAS;        // both CTAs of a pair walk the same tiles
   const int tile_step = gridDim.x / CTAS;
@@ -164,11 +176,13 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_kernel(const __grid_cons
     if (lane == 0) {
       uint32_t it = 0;
       bool ok = true;
-      for (int tile = first_tile; tile < num_tiles && ok; tile += tile_step) {
+      for (int work = first_tile; work < num_work && ok; work += tile_step) {
+        const int tile = SPLIT ? work / n_splits : work, split = SPLIT ? work - tile * n_splits : 0;
         int mg, nb;
         tile_coords(p.reverse ? num_tiles - 1 - tile : tile, p.m_blocks, p.n_blocks, mg, nb);
         const int mb = mg * CTAS + cta_rank;       // this CTA's 128-row block
-        for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
+        const int kb0 = split * kb_per_split, kb1 = SPLIT ? min(p.k_blocks, kb0 + kb_per_split) : p.k_blocks;
+        for (int kb = kb0; kb < kb1; ++kb, ++it) {
           const int s = it % kStages;
           const uint32_t ph = (it / kStages) & 1u;
           if (!mbar_wait(&empty_bar[s], ph ^ 1u, abort_flag)) { ok = false; break; }
@@ -220,17 +234,19 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_kernel(const __grid_cons
       constexpr uint32_t idesc = make_idesc_bf16(kBM * CTAS, kBN, 0, 0);
       uint32_t it = 0, tcount = 0;
       bool ok = true;
-      for (int tile = first_tile; tile < num_tiles && ok; tile += tile_step, ++tcount) {
+      for (int work = first_tile; work < num_work && ok; work += tile_step, ++tcount) {
         const uint32_t acc = tcount % kAccBuffers;
         const uint32_t acc_ph = (tcount / kAccBuffers) & 1u;
         if (!mbar_wait(&acc_empty[acc], acc_ph ^ 1u, abort_flag)) { ok = false; break; }
         tc_fence_after_sync();
         const uint32_t tmem_d = tmem_base + acc * kBN;
-        for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
+        const int split = SPLIT ? work % n_splits : 0;
+        const int kb0 = split * kb_per_split, kb1 = SPLIT ? min(p.k_blocks, kb0 + kb_per_split) : p.k_blocks;
+        for (int kb = kb0; kb < kb1; ++kb, ++it) {
           const int s = it % kStages;
           const uint32_t ph = (it / kStages) & 1u;
           if (!mbar_wait(&full_bar[s], ph, abort_flag)) { ok = false; break; }
-          if (tcount == 0 && kb == 0) GEMM_TL(3);
+          if (tcount == 0 && kb == kb0) GEMM_TL(3);
           tc_fence_after_sync();
           const uint32_t a_addr = smem_u32(smem + s * kStageBytes);
           const uint32_t b_addr = a_addr + kABytes * KD;
@@ -245,9 +261,9 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_kernel(const __grid_cons
 #pragma unroll
                 for (int h = 0; h < NW; ++h)   // second accumulator: the next 128 weight rows of each CTA
                   umma_bf16_ss_pair(tmem_d + h * kBN, adesc + 2 * k, bdesc + 2 * k + h * (kBAtom * KD / 16), idesc,
-                                    (kb | a | k) != 0);
+                                    ((kb - kb0) | a | k) != 0);
               } else {
-                umma_bf16_ss(tmem_d, adesc + 2 * k, bdesc + 2 * k, idesc, (kb | a | k) != 0);
+                umma_bf16_ss(tmem_d, adesc + 2 * k, bdesc + 2 * k, idesc, ((kb - kb0) | a | k) != 0);
               }
             }
           }
@@ -275,7 +291,8 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_kernel(const __grid_cons
         if (CTAS == 2) mbar_arrive_cluster_relaxed(&acc_empty[acc], 0); else mbar_arrive(&acc_empty[acc]);
       }
     };
-    for (int tile = first_tile; tile < num_tiles && ok; tile += tile_step, ++tcount) {
+    for (int work = first_tile; work < num_work && ok; work += tile_step, ++tcount) {
+      const int tile = SPLIT ? work / n_splits : work, split = SPLIT ? work - tile * n_splits : 0;
       int mg, nb;
       tile_coords(p.reverse ? num_tiles - 1 - tile : tile, p.m_blocks, p.n_blocks, mg, nb);
       const int mb = mg * CTAS + cta_rank;
@@ -289,7 +306,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_kernel(const __grid_cons
 #pragma unroll
           for (int h = 0; h < NW; ++h) {
             const int col = nb * kTileN + h * 256 + ew * 32 + lane;
-            sbias[h * 256 + ew * 32 + lane] = col < p.N ? __bfloat162float(p.bias[col]) : 0.f;
+            sbias[h * 256 + ew * 32 + lane] = (col < p.N && split == 0) ? __bfloat162float(p.bias[col]) : 0.f;
           }
           __syncwarp();
           if (lane == 0) mbar_arrive(&bias_bar[acc]);
@@ -337,16 +354,22 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_kernel(const __grid_cons
           if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
           __syncwarp();
         };
+        // where the sub-tiles go: the output (reduce-added into the fp32 residual stream), or, for the bare partial sums
+        // of a later split, this split's region of the scratch matrix (plain stores)
+        const bool later_split = SPLIT && OUT == OUT_F32 && split > 0;
+        const uint64_t out_map = reinterpret_cast<uint64_t>(later_split ? &p.tma_part : &p.tma_out);
+        const int out_y = later_split ? (split - 1) * p.part_rows + ycoord : ycoord;
+        const bool out_reduce = OUT == OUT_F32 && p.resid != nullptr && !later_split;
         auto store_subtile = [&](int x) { // one TMA store / reduce-add of the 32-row staging buffer at column x
           fence_proxy_async_smem();
           __syncwarp();
           if (lane == 0) {
-            if (OUT == OUT_F32 && p.resid != nullptr) {
+            if (out_reduce) {
               asm volatile("cp.reduce.async.bulk.tensor.2d.global.shared::cta.add.bulk_group [%0, {%2, %3}], [%1];"
-                           ::"l"(reinterpret_cast<uint64_t>(&p.tma_out)), "r"(smem_u32(stage)), "r"(x), "r"(ycoord) : "memory");
+                           ::"l"(out_map), "r"(smem_u32(stage)), "r"(x), "r"(out_y) : "memory");
             } else {
               asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
-                           ::"l"(reinterpret_cast<uint64_t>(&p.tma_out)), "r"(smem_u32(stage)), "r"(x), "r"(ycoord) : "memory");
+                           ::"l"(out_map), "r"(smem_u32(stage)), "r"(x), "r"(out_y) : "memory");
             }
             asm volatile("cp.async.bulk.commit_group;" ::: "memory");
           }

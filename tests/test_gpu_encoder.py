@@ -80,3 +80,51 @@ def test_invalid_arguments_are_rejected_before_launch():
     with pytest.raises(P.EasError) as e:
         enc.status()
     assert e.value.status == 7
+
+
+def test_split_k_is_deterministic_budget_independent_and_optional():
+    """Latency path: small micro-batches split the K loop of the residual GEMMs (eas_encoder_set_split_k, off by default).  The result must not depend
+    on sm_budget or on the run, must stay within the oracle tolerance, and with the mode off an item's embeddings are
+    bit-identical whatever it is packed with."""
+    cfg = S.get_config("c1", n_layers=3)
+    w, enc = _make(cfg)
+    shapes = [(1, 336, 336)] * 2                                  # 1154 tokens: fc2 (K = 4096) splits, proj does not
+    items = S.make_items(cfg, shapes, seed=2100)
+    ref, _, _ = O.encode_microbatch(cfg, w, items)
+    enc.set_split_k(True)
+    got, a = G.run_gpu(enc, cfg, items)
+    G.assert_parity(got, ref, "split K")
+    _, b = G.run_gpu(enc, cfg, items)
+    assert torch.equal(a, b)
+    for budget in (20, 37, 111):
+        _, c = G.run_gpu(enc, cfg, items, sm_budget=budget)
+        assert torch.equal(a, c), budget
+    enc.set_split_k(False)
+    got_off, off = G.run_gpu(enc, cfg, items)
+    G.assert_parity(got_off, ref, "split K off")
+    assert not torch.equal(a, off)                                # the mode did something (another summation order)
+    assert float((a.float() - off.float()).abs().max()) < 0.05
+    rows = off.shape[0] // 2
+    _, alone = G.run_gpu(enc, cfg, [items[1]])
+    assert torch.equal(off[rows:], alone)                         # off: item alone == item packed
+    big = items + S.make_items(cfg, [(1, 336, 336)] * 4, seed=2101)    # 3462 tokens: no split either way
+    _, packed = G.run_gpu(enc, cfg, big)
+    assert torch.equal(packed[rows:2 * rows], alone)
+    enc.set_split_k(True)
+    _, packed_on = G.run_gpu(enc, cfg, big)
+    assert torch.equal(packed_on, packed)
+
+
+@pytest.mark.parametrize("case", ["c1_2layers", "c2_2layers", "c3_2layers", "c4_2layers"])
+def test_split_k_parity_all_families(case):
+    """The small cases of every family with split K on (RMSNorm and LayerNorm, SwiGLU and GELU MLPs, d = 1024 and 1280)."""
+    name, over, shapes = CASES[case]
+    cfg = S.get_config(name, **over)
+    w, enc = _make(cfg, "sharp")
+    enc.set_split_k(True)
+    items = S.make_items(cfg, shapes, seed=2300 + len(shapes))
+    ref, _, _ = O.encode_microbatch(cfg, w, items)
+    got, dev = G.run_gpu(enc, cfg, items)
+    G.assert_parity(got, ref, case + " split K")
+    _, again = G.run_gpu(enc, cfg, items, sm_budget=37)
+    assert torch.equal(dev, again)
