@@ -28,9 +28,11 @@ from . import serving as SV  # noqa: E402
 class EncodeWorker:
     """One encoder handle plus cached per-batch-size inputs; measures the device time of a forward pass."""
 
-    def __init__(self, config: str):
+    def __init__(self, config: str, split_k: bool = False):
         self.cfg = S.get_config(config)
         self.enc = B.Encoder(self.cfg, B.weights_to_device(S.make_weights(self.cfg)))
+        if split_k:                      # latency path for the small micro-batches of a lightly loaded worker
+            self.enc.set_split_k(True)
         self._inputs = {}
 
     def _batch(self, n: int):
@@ -129,8 +131,9 @@ def main():
     ap.add_argument("--offload", type=float, default=0.7)
     ap.add_argument("--arrival-cv", type=float, default=1.0)
     ap.add_argument("--no-table", action="store_true")
+    ap.add_argument("--split-k", action="store_true", help="latency path: split K in micro-batches with few tiles")
     a = ap.parse_args()
-    w = EncodeWorker(a.config)
+    w = EncodeWorker(a.config, split_k=a.split_k)
     sm_total = torch.cuda.get_device_properties(0).multi_processor_count
     ce, b_sat, curve = profile_encode_capacity(w)
     print(json.dumps({"capacity_items_per_s": ce, "saturation_batch": b_sat, "curve": curve}))
