@@ -11,8 +11,10 @@
 //
 // The grid is `sm_budget` CTAs (one per SM: the shared-memory request excludes a second resident
 // CTA) and each CTA walks tiles  blockIdx.x, blockIdx.x + gridDim.x, ...  in a fixed order; every output element is
-// accumulated over K in the same order whatever the tile shape, so the result never depends on the budget: no split-K,
-// no atomics on the accumulation (the fp32 residual update is one add per element).
+// accumulated over K in the same order whatever the tile shape, so the result never depends on the budget: no atomics on
+// the accumulation (the fp32 residual update is one add per element).  The SPLIT instantiations (opt-in, small
+// micro-batches) share a tile's K range among CTAs: the later splits store bare partial sums that the following
+// normalisation kernel adds in a fixed order, so that mode is deterministic and budget-independent as well.
 #pragma once
 #include "ptx.cuh"
 
