@@ -116,3 +116,36 @@ def test_invalid_input_in_graph_mode_reports_the_ordinary_error_and_leaves_the_s
         enc.status(side)
     assert np.isfinite(good.float().cpu().numpy()).all()
     assert enc.graph_stats()["captures"] == 1
+
+
+def test_graph_replay_with_split_k_is_bit_identical():
+    """The two halves of the latency path together: split K (partial sums added by the following normalisation) inside
+    captured and replayed forward passes, and through the allocation-free entry point."""
+    shapes = [(1, 336, 336)]
+    P, cfg, enc, items, data, offsets, cu = _setup("c1", shapes, seed=23)
+    cu_dev = torch.from_numpy(cu).cuda()
+    plain = enc.encode_microbatch(data, shapes, offsets, cu, cu_seqlens_dev=cu_dev)
+    enc.status()
+    enc.set_split_k(True)
+    ref = enc.encode_microbatch(data, shapes, offsets, cu, cu_seqlens_dev=cu_dev)
+    enc.status()
+    # another summation order: a few bf16 last-place differences after 24 layers, nothing more
+    assert not torch.equal(ref, plain)
+    assert float((ref.float() - plain.float()).abs().max()) <= 2.0 ** -6 * float(plain.float().abs().max())
+    ws = torch.empty(enc.workspace_bytes(int(cu[-1]), 1) + 1024, dtype=torch.uint8, device="cuda")
+    out = torch.zeros_like(ref)
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    enc.set_graph_mode(True)
+    with torch.cuda.stream(side):
+        for it in range(3):
+            out.zero_()
+            enc.encode_microbatch(data, shapes, offsets, cu, cu_seqlens_dev=cu_dev, out=out, workspace=ws, stream=side)
+            enc.status(side)
+            assert torch.equal(out, ref), f"call {it}"
+        assert enc.graph_stats()["hits"] == 2
+    enc.set_graph_mode(False)
+    out.zero_()
+    enc.encode_microbatch_static(data, shapes, offsets, cu, cu_dev, out)
+    enc.status()
+    assert torch.equal(out, ref)
