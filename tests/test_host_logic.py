@@ -94,7 +94,7 @@ def test_generators_are_seeded_and_bf16_exact():
     assert S.tokens_per_item(S.get_config("c4"), (3000, 128, 1)) == 1500
 
 
-def test_bench_flop_model_matches_the_survey_totals():
+def test_bench_flop_model_matches_the_per_item_totals():
     sys.path.insert(0, ROOT)
     import bench
     c1 = S.get_config("c1")
