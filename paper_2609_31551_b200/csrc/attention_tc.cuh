@@ -19,7 +19,9 @@
 // P = exp2((s - m) * scale) as bf16 into shared memory (K-major, 128-byte swizzle: the A operand of P V).
 // The reference maximum only moves when the row maximum grows by more than 2^8 in the exponent; then the
 // thread rescales its O row in TMEM.  Final O / l is written as bf16.
-// Persistent: gridDim.x = sm_budget CTAs walk units blockIdx.x, +gridDim.x, ... in a fixed order.
+// Persistent: gridDim.x = sm_budget CTAs; the units are dealt to them in rounds of gridDim.x, alternate rounds in
+// opposite directions (the host sorts the units by decreasing cost: a fixed direction would hand CTA 0 the costliest
+// unit of every round).
 #pragma once
 #include "ptx.cuh"
 
@@ -323,6 +325,11 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_tc_kernel(const __grid_con
   pdl_launch_dependents();
   pdl_wait();
 
+  // this CTA's unit of a round; increasing in `round`
+  auto unit_at = [&](uint32_t round) -> int {
+    const int g = static_cast<int>(gridDim.x), b = static_cast<int>(blockIdx.x);
+    return static_cast<int>(round) * g + ((round & 1u) ? g - 1 - b : b);
+  };
   auto q_tile = [&](int buf, int t) { return smem + L::kQOff + (buf * 2 + t) * L::kTileBytes; };
   auto k_tile = [&](int s) { return smem + L::kKvOff + s * L::kStageBytes; };
   auto v_tile = [&](int s) { return smem + L::kKvOff + s * L::kStageBytes + L::kKTileBytes; };
@@ -335,7 +342,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_tc_kernel(const __grid_con
       uint32_t kv_it = 0, u_cnt = 0;
       bool ok = true;
       int cursor = 0;
-      for (int unit = blockIdx.x; unit < p.total_units && ok; unit += gridDim.x, ++u_cnt) {
+      for (int unit = unit_at(0); unit < p.total_units && ok; unit = unit_at(++u_cnt)) {
         const UnitInfo u = decode_unit<DUAL, L::kKeys>(p, unit, cursor);
         const int qb = u_cnt & 1;
         if (!mbar_wait(&q_empty[qb], ((u_cnt >> 1) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
@@ -452,10 +459,10 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_tc_kernel(const __grid_con
         };
         auto next_tile = [&](Pos& c) {
           ++c.j; ++c.g;
-          if (c.j >= c.n_kv) { c.unit += gridDim.x; ++c.ucnt; enter_unit(c); }
+          if (c.j >= c.n_kv) { ++c.ucnt; c.unit = unit_at(c.ucnt); enter_unit(c); }
         };
         Pos pc;                                      // in-order position: every tile is visited
-        pc.unit = blockIdx.x; pc.ucnt = 0; pc.g = 0; pc.hint = 0; pc.end = false;
+        pc.unit = unit_at(0); pc.ucnt = 0; pc.g = 0; pc.hint = 0; pc.end = false;
         enter_unit(pc);
         bool s_issued = false;                       // S of the own tile at pc is already in flight
         uint32_t q_seen = 0;                         // units before this one have had their Q seen landing by this thread
@@ -514,11 +521,11 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_tc_kernel(const __grid_con
         bool pre_issued[2] = {false, false};       // S(w, 0) of this unit was already issued at the end of the previous one
         int cursor = 0;
         UnitInfo un = decode_unit<DUAL, L::kKeys>(p, min(static_cast<int>(blockIdx.x), p.total_units - 1), cursor);
-        for (int unit = blockIdx.x; unit < p.total_units && ok; unit += gridDim.x, ++u_cnt) {
+        for (int unit = unit_at(0); unit < p.total_units && ok; unit = unit_at(++u_cnt)) {
           const UnitInfo u = un;
           const int qb = u_cnt & 1;
-          const bool has_next = unit + static_cast<int>(gridDim.x) < p.total_units;
-          if (has_next) un = decode_unit<DUAL, L::kKeys>(p, unit + gridDim.x, cursor);
+          const bool has_next = unit_at(u_cnt + 1) < p.total_units;
+          if (has_next) un = decode_unit<DUAL, L::kKeys>(p, unit_at(u_cnt + 1), cursor);
           if (!mbar_wait(&q_full[qb], (u_cnt >> 1) & 1u, abort_flag)) { ok = false; break; }
           // K/V tile of warpgroup w at ring position kv_it: shared by both warpgroups, or (dual-head unit) one each
           const uint32_t step = 1 + u.dual;
@@ -660,12 +667,13 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_tc_kernel(const __grid_con
 
     int cursor = 0;
     UnitInfo u_next = decode_unit<DUAL, L::kKeys>(p, min(static_cast<int>(blockIdx.x), p.total_units - 1), cursor);
-    for (int unit = blockIdx.x; unit < p.total_units && ok; unit += gridDim.x) {
+    uint32_t round = 0;
+    for (int unit = unit_at(0); unit < p.total_units && ok; unit = unit_at(++round)) {
       const UnitInfo u = u_next;
       ATTN_STAMP_PREV(10);
-      const bool has_next = unit + static_cast<int>(gridDim.x) < p.total_units;
+      const bool has_next = unit_at(round + 1) < p.total_units;
       if (w >= u.n_q) {                             // this warpgroup has no tile in the unit
-        if (has_next) u_next = decode_unit<DUAL, L::kKeys>(p, unit + gridDim.x, cursor);
+        if (has_next) u_next = decode_unit<DUAL, L::kKeys>(p, unit_at(round + 1), cursor);
         if (pend && !flush_output()) { ok = false; break; }
         continue;
       }
@@ -797,7 +805,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_tc_kernel(const __grid_con
         if (lane == 0) mbar_arrive(&p_ready[w]);
         ATTN_STAMP(6);
         // decode the following unit here: the warp now waits for the issuer anyway
-        if (j == 0 && has_next) u_next = decode_unit<DUAL, L::kKeys>(p, unit + gridDim.x, cursor);
+        if (j == 0 && has_next) u_next = decode_unit<DUAL, L::kKeys>(p, unit_at(round + 1), cursor);
       }
       if (!ok) break;
       pend = true;                                  // written later, see flush_output
