@@ -102,7 +102,7 @@ def tokens_per_item(cfg: dict, shape) -> int:
     """Encoder tokens of one item.  shape = (frames, height, width); audio: (n_frames, n_mel, 1)."""
     f, h, w = (int(v) for v in shape)
     if cfg["family"] == FAMILY_AUDIO_CONV:
-        return f // 2
+        return (f + 1) // 2         # k=3, stride 2, padding 1: floor((f - 1) / 2) + 1 output frames
     P = cfg["patch"]
     return (f // cfg["temporal_patch"]) * (h // P) * (w // P) + (1 if cfg["has_cls"] else 0)
 

@@ -46,6 +46,7 @@ enum { EAS_NORM_LAYERNORM = 0, EAS_NORM_RMSNORM = 1 };
 enum { EAS_MLP_GELU = 0, EAS_MLP_SWIGLU = 1 };
 enum { EAS_POS_TABLE = 0, EAS_POS_ROPE_2D = 1 };
 enum { EAS_HEAD_NONE = 0, EAS_HEAD_MLP_PROJECTOR = 1, EAS_HEAD_MERGER_2X2 = 2 };
+enum { EAS_OUT_BF16 = 0, EAS_OUT_FP32 = 1 };
 enum { EAS_MAX_ITEMS = 128 }; /* items per micro-batch */
 
 /* Architecture record (plain data, copied at create).  Encoder = embedding front end, n_layers
@@ -70,6 +71,9 @@ typedef struct {
   int32_t head;           /* EAS_HEAD_* */
   int32_t d_head_hidden;  /* hidden width of the connector MLP */
   int32_t d_out;          /* embedding width delivered to the LLM */
+  int32_t out_dtype;      /* EAS_OUT_BF16 (default): out_embeddings is bf16.  EAS_OUT_FP32: the last kernel (final norm or
+                             the connector's second GEMM) writes its fp32 result unrounded, out_embeddings is fp32
+                             [out_rows, d_out]: for consumers that want the embeddings without the 2^-9 output rounding */
 } eas_arch_config;
 
 /* One named weight tensor in device memory, bf16.
@@ -99,7 +103,8 @@ typedef struct {
 typedef struct {
   const void* data;               /* device, bf16, items back to back.  Image [C,H,W]; clip [F,C,H,W]; audio [frames, mel] */
   int32_t n_items;                /* 1..EAS_MAX_ITEMS */
-  const int32_t* item_shape;      /* host [n_items][3]: (frames, height, width); audio: (n_frames, n_mel, 1) */
+  const int32_t* item_shape;      /* host [n_items][3]: (frames, height, width); audio: (n_frames, n_mel, 1), any
+                                     n_frames >= 1: the stride-2 convolution yields ceil(n_frames / 2) tokens */
   const int64_t* item_offset;     /* host [n_items]: element offset of each item in data */
   const int32_t* cu_seqlens_host; /* host [n_items+1]: prefix sums of ENCODER tokens per item (after patching or
                                      convolution, CLS included); checked against item_shape */
@@ -128,7 +133,8 @@ int64_t eas_encoder_out_rows(const eas_encoder* enc, const int32_t* cu_seqlens_h
  *   raises EAS_ERR_DEVICE_CHECK at the next eas_encoder_status).  Items never attend across each other.
  * sm_budget: number of SMs every kernel of this call may occupy, 1..SM count; 0 = all.
  * stream: a cudaStream_t (NULL = legacy default stream).
- * out_embeddings: device bf16 [out_rows, d_out]; rows of item i start at the sum of earlier items' rows.
+ * out_embeddings: device bf16 (fp32 with EAS_OUT_FP32) [out_rows, d_out]; rows of item i start at the sum of earlier
+ *   items' rows.
  * Errors (nothing launched): INVALID_ARG (null pointers, n_items out of range, non-monotone cu_seqlens,
  *   sizes not multiples of the patch / merge / temporal patch, tokens inconsistent with shapes, more tokens
  *   than position rows, sm_budget out of range), WORKSPACE. */
@@ -143,8 +149,12 @@ eas_status eas_encode_microbatch(eas_encoder* enc, const eas_packed_inputs* in, 
  * EAS_STATIC_WORKSPACE_BYTES that is part of the library image, so the call itself allocates nothing (no cudaMalloc,
  * cudaFree, or allocating library routine).  in->workspace and in->workspace_bytes are ignored; the caller still
  * provides data, cu_seqlens and out_embeddings.
- *  - Limit: the micro-batch must fit the built-in scratch (about 20 KB per token for a d=256 model, 90 KB per token
- *    for d=1280); a larger one is rejected with EAS_ERR_WORKSPACE and a message that states both sizes.
+ *  - Limit: the micro-batch must fit the built-in scratch.  The forward pass needs about
+ *    14 * d_model + 2 * d_mlp + 2 * (patch elements, padded to 64) bytes per encoder token (fp32 residual stream, bf16
+ *    normalised rows, Q|K|V, attention output, MLP activation, patch operand), i.e. about 7 KB per token for d_model = 256
+ *    with d_mlp = 1024 and about 30 KB per token for d_model = 1280 with d_mlp = 5120; eas_encoder_workspace_bytes()
+ *    gives the exact figure.  32 MiB hold about 4600 tokens of the former and 1100 of the latter.  A larger micro-batch
+ *    is rejected with EAS_ERR_WORKSPACE and a message that states both sizes.
  *  - Cost: every GPU on which this library is loaded holds the array until the process exits.
  *  - The first call on each device looks up the array's device address (cudaGetSymbolAddress, with that device
  *    current).  Make that first call before starting any stream capture.
@@ -237,6 +247,15 @@ void eas_encoder_destroy(eas_encoder* enc);
 eas_status eas_kernel_gemm(const void* A, const void* W, const void* bias, void* out, const float* resid,
                            int32_t M, int32_t N, int32_t K, int32_t act, int32_t out_fp32, int32_t sm_budget,
                            void* stream, uint32_t* status_dev);
+
+/* The same call with the tile shape fixed instead of chosen by the launcher's cost model: 0 = choose (as above),
+ * 1 = one CTA per 128x256 tile, 2 = a CTA pair per 256x256 tile, 3 = a CTA pair per 256x512 tile (needs N % 512 == 0,
+ * act 0 or 1; EAS_ERR_UNSUPPORTED otherwise).  All shapes accumulate over K in the same order, so their results are
+ * bit-identical; the tests use this to check exactly that.  With sm_budget 1 only shape 1 exists and the argument is
+ * ignored. */
+eas_status eas_kernel_gemm_tile(const void* A, const void* W, const void* bias, void* out, const float* resid,
+                                int32_t M, int32_t N, int32_t K, int32_t act, int32_t out_fp32, int32_t sm_budget,
+                                void* stream, uint32_t* status_dev, int32_t tile_shape);
 
 /* y[rows,d] = norm(x[rows,d]): kind 0 LayerNorm (gamma, beta), 1 RMSNorm (gamma), 2 plain cast.  x device fp32;
  * gamma/beta device bf16; y device bf16 (out_fp32 = 0) or fp32.  d % 128 == 0, d <= 2048. */

@@ -16,7 +16,7 @@ STATUS_NAMES = {0: "EAS_OK", 1: "EAS_ERR_INVALID_ARG", 2: "EAS_ERR_UNSUPPORTED",
 EXPORTED_SYMBOLS = [
     "eas_encoder_create", "eas_encoder_weight_arena_bytes", "eas_encoder_workspace_bytes", "eas_encoder_out_rows",
     "eas_encode_microbatch", "eas_encode_microbatch_static", "eas_encoder_status", "eas_encoder_last_launch_count", "eas_encoder_set_attention_impl",
-    "eas_encoder_set_graph_mode", "eas_encoder_graph_stats", "eas_encoder_enable_timing", "eas_encoder_timing_read", "eas_last_error", "eas_encoder_destroy", "eas_kernel_gemm", "eas_kernel_norm", "eas_kernel_attention",
+    "eas_encoder_set_graph_mode", "eas_encoder_graph_stats", "eas_encoder_enable_timing", "eas_encoder_timing_read", "eas_last_error", "eas_encoder_destroy", "eas_kernel_gemm", "eas_kernel_gemm_tile", "eas_kernel_norm", "eas_kernel_attention",
     "eas_encoder_set_split_k", "eas_sm_partition_create", "eas_sm_partition_sm_count", "eas_sm_partition_stream", "eas_sm_partition_destroy",
 ]
 
@@ -33,7 +33,7 @@ class ArchConfig(C.Structure):
                 ("in_channels", C.c_int32), ("patch", C.c_int32), ("temporal_patch", C.c_int32),
                 ("has_cls", C.c_int32), ("embed_norm", C.c_int32), ("final_norm", C.c_int32), ("pos", C.c_int32),
                 ("max_pos", C.c_int32), ("rope_theta", C.c_float), ("head", C.c_int32),
-                ("d_head_hidden", C.c_int32), ("d_out", C.c_int32)]
+                ("d_head_hidden", C.c_int32), ("d_out", C.c_int32), ("out_dtype", C.c_int32)]
 
 
 class Tensor(C.Structure):
@@ -95,6 +95,8 @@ def load_library():
     lib.eas_kernel_gemm.restype = C.c_int
     lib.eas_kernel_gemm.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32,
                                     C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p]
+    lib.eas_kernel_gemm_tile.restype = C.c_int
+    lib.eas_kernel_gemm_tile.argtypes = lib.eas_kernel_gemm.argtypes + [C.c_int32]
     lib.eas_kernel_norm.restype = C.c_int
     lib.eas_kernel_norm.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32,
                                     C.c_float, C.c_int32, C.c_int32, C.c_void_p]
@@ -127,7 +129,7 @@ def _stream_ptr(stream) -> int:
 def arch_struct(cfg: dict) -> ArchConfig:
     a = ArchConfig()
     for name, _ in ArchConfig._fields_:
-        setattr(a, name, cfg[name])
+        setattr(a, name, cfg.get("out_dtype", 0) if name == "out_dtype" else cfg[name])
     return a
 
 
@@ -224,7 +226,8 @@ class Encoder:
         ws_bytes = workspace.numel() - (ws_ptr - workspace.data_ptr())
         if out is None:
             rows = self.out_rows(cu)
-            out = torch.empty((max(rows, 0), self.cfg["d_out"]), dtype=torch.bfloat16, device=data.device)
+            out = torch.empty((max(rows, 0), self.cfg["d_out"]), device=data.device,
+                              dtype=torch.float32 if self.cfg.get("out_dtype", 0) else torch.bfloat16)
         pin = PackedInputs(data.data_ptr(), n, shp.ctypes.data_as(C.POINTER(C.c_int32)),
                            offs.ctypes.data_as(C.POINTER(C.c_int64)), cu.ctypes.data_as(C.POINTER(C.c_int32)),
                            ws_ptr, ws_bytes)
@@ -313,9 +316,10 @@ class SmPartition:
             pass
 
 
-def kernel_gemm(A, W, bias, act=0, out_fp32=False, resid=None, sm_budget=0, stream=None, out=None, status=None):
-    """eas_kernel_gemm on device tensors.  Returns (out, device status word).  `status` (device int32, zeroed by the
-    caller) can be passed in so that a call allocates nothing."""
+def kernel_gemm(A, W, bias, act=0, out_fp32=False, resid=None, sm_budget=0, stream=None, out=None, status=None,
+                tile_shape=0):
+    """eas_kernel_gemm (eas_kernel_gemm_tile when tile_shape != 0) on device tensors.  Returns (out, device status
+    word).  `status` (device int32, zeroed by the caller) can be passed in so that a call allocates nothing."""
     lib = load_library()
     M, K = A.shape
     N = W.shape[0]
@@ -323,9 +327,13 @@ def kernel_gemm(A, W, bias, act=0, out_fp32=False, resid=None, sm_budget=0, stre
         out = torch.empty((M, N // 2 if act == 2 else N), dtype=torch.float32 if out_fp32 else torch.bfloat16, device=A.device)
     if status is None:
         status = torch.zeros(4, dtype=torch.int32, device=A.device)
-    _check(lib.eas_kernel_gemm(A.data_ptr(), W.data_ptr(), bias.data_ptr(), out.data_ptr(),
-                               resid.data_ptr() if resid is not None else None, M, N, K, act, int(out_fp32), sm_budget,
-                               _stream_ptr(stream), status.data_ptr()))
+    args = (A.data_ptr(), W.data_ptr(), bias.data_ptr(), out.data_ptr(),
+            resid.data_ptr() if resid is not None else None, M, N, K, act, int(out_fp32), sm_budget,
+            _stream_ptr(stream), status.data_ptr())
+    if tile_shape:
+        _check(lib.eas_kernel_gemm_tile(*args, tile_shape))
+    else:
+        _check(lib.eas_kernel_gemm(*args))
     return out, status
 
 

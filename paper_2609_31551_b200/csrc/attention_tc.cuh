@@ -15,10 +15,11 @@
 //   warps 4..7   softmax warpgroup of tile A: one thread per query row
 //   warps 8..11  softmax warpgroup of tile B
 //
-// A softmax thread reads its row of S from TMEM, keeps a running reference maximum m and sum l, writes
-// P = exp2((s - m) * scale) as bf16 into shared memory (K-major, 128-byte swizzle: the A operand of P V).
-// The reference maximum only moves when the row maximum grows by more than 2^8 in the exponent; then the
-// thread rescales its O row in TMEM.  Final O / l is written as bf16.
+// A softmax thread reads its row of S from TMEM, keeps a running reference maximum m and sum l, and writes
+// P = exp2((s - m) * scale) as bf16 back into tensor memory (columns of its own: the A operand of P V is read from
+// there; the PT = false instantiation, kept as a cross-check, stages P in shared memory instead, K-major with
+// 128-byte swizzle).  The reference maximum only moves when the row maximum grows by more than 2^8 in the exponent;
+// then the thread rescales its O row in TMEM.  Final O / l is written as bf16.
 // Persistent: gridDim.x = sm_budget CTAs; the units are dealt to them in rounds of gridDim.x, alternate rounds in
 // opposite directions (the host sorts the units by decreasing cost: a fixed direction would hand CTA 0 the costliest
 // unit of every round).

@@ -144,6 +144,7 @@ constexpr size_t kMaxGraphs = 16;
 
 struct eas_encoder {
   eas_arch_config cfg;
+  int device = 0;             // ordinal of the device that was current at create: weights, tensor maps and kernel attributes belong to it
   int sm_count = 0;
   int hd = 0;
   int embed_k = 0, embed_k_pad = 0;
@@ -211,6 +212,7 @@ static eas_status check_cfg(const eas_arch_config* c) {
     return fail(EAS_ERR_UNSUPPORTED, "connector widths must be multiples of 64 (hidden) and 32 (out)");
   if (c->head == EAS_HEAD_NONE && c->d_out != c->d_model) return fail(EAS_ERR_INVALID_ARG, "d_out must equal d_model without a head");
   if (c->head == EAS_HEAD_MLP_PROJECTOR && c->final_norm) return fail(EAS_ERR_UNSUPPORTED, "projector after a final norm");
+  if (c->out_dtype != EAS_OUT_BF16 && c->out_dtype != EAS_OUT_FP32) return fail(EAS_ERR_INVALID_ARG, "unknown out_dtype %d", c->out_dtype);
   return EAS_OK;
 }
 
@@ -280,14 +282,19 @@ static eas_status relayout(bf16* dst, const bf16* src, const bf16* src2, long lo
 struct OncePerDevice {
   std::mutex m;
   bool done[64] = {};
-  // true exactly once per device ordinal (false for ordinals past the table: the attribute is then set every time)
+  // true until settled() has been called with this device current (always true for ordinals past the table: the
+  // attribute is then set every time).  A failed attribute call returns before settled(), so the next launch retries.
   bool first() {
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return true;
     std::lock_guard<std::mutex> lock(m);
-    if (done[dev]) return false;
+    return !done[dev];
+  }
+  void settled() {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return;
+    std::lock_guard<std::mutex> lock(m);
     done[dev] = true;
-    return true;
   }
 };
 
@@ -347,13 +354,24 @@ static eas_status set_kernel_attributes() {
   return EAS_OK;
 }
 
+// the GEMM kernels' attributes, once per device (create-time and the single-kernel entry point both come through here)
+static eas_status set_kernel_attributes_once() {
+  static OncePerDevice once;
+  if (once.first()) {
+    EAS_TRY(set_kernel_attributes());
+    once.settled();
+  }
+  return EAS_OK;
+}
+
 // shared memory requested by the light kernels: more than half an SM's capacity, so that a second CTA
 // can never be co-resident and a grid of B CTAs occupies B SMs
 constexpr int kOnePerSmSmem = 120 * 1024;
 
-static eas_status device_check(int* sm_count) {
+static eas_status device_check(int* sm_count, int* device = nullptr) {
   int dev = 0;
   CUDA_TRY(cudaGetDevice(&dev));
+  if (device != nullptr) *device = dev;
   int major = 0, minor = 0, sms = 0;
   CUDA_TRY(cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev));
   CUDA_TRY(cudaDeviceGetAttribute(&minor, cudaDevAttrComputeCapabilityMinor, dev));
@@ -372,9 +390,9 @@ extern "C" eas_status eas_encoder_create(const eas_arch_config* arch, const eas_
   const size_t need = eas_encoder_weight_arena_bytes(arch);
   if (weights->arena == nullptr || weights->arena_bytes < need)
     return fail(EAS_ERR_WORKSPACE, "weight arena too small: %zu bytes given, %zu needed", weights->arena_bytes, need);
-  int sm_count = 0;
-  EAS_TRY(device_check(&sm_count));
-  EAS_TRY(set_kernel_attributes());
+  int sm_count = 0, device = 0;
+  EAS_TRY(device_check(&sm_count, &device));
+  EAS_TRY(set_kernel_attributes_once());
 
   WeightIndex wi;
   for (int i = 0; i < weights->n_tensors; ++i) {
@@ -384,6 +402,7 @@ extern "C" eas_status eas_encoder_create(const eas_arch_config* arch, const eas_
   eas_encoder* e = new eas_encoder();
   std::unique_ptr<eas_encoder> guard(e);
   e->cfg = *arch;
+  e->device = device;
   e->sm_count = sm_count;
   const eas_arch_config& c = e->cfg;
   const int d = c.d_model, I = c.d_mlp;
@@ -578,8 +597,14 @@ extern "C" int64_t eas_encoder_out_rows(const eas_encoder* enc, const int32_t* c
 }
 
 // ------------------------------------------------------------------------------------ launch helpers
-// Every per-call kernel is launched with programmatic stream serialization: it may be set up while its
-// predecessor in the stream drains and waits (griddepcontrol.wait) before touching any data.
+// A call that owns the whole device launches its kernels with programmatic stream serialization: a kernel may be set
+// up while its predecessor in the stream drains, and waits (griddepcontrol.wait) before touching any data.  A call on
+// a SHARE of the SMs (Section 3.4) must not: its grids are persistent (all CTAs resident at once), so a dependent
+// kernel would be released the moment its predecessor started, its CTAs would settle on SMs outside the share and
+// sit there holding shared memory and tensor memory while they wait -- exactly the SMs the co-resident worker was
+// promised.  Without the attribute a kernel starts when its predecessor has finished, and at most `sm_budget` SMs
+// hold a CTA of this call at any time.  Set by every entry point before its first launch (per host thread).
+static thread_local bool g_overlap_launches = true;
 template <typename Params>
 static eas_status launch_kernel(void (*kern)(Params), int grid, int block, size_t smem, cudaStream_t stream, const Params& params,
                                 int cluster = 1) {
@@ -590,9 +615,11 @@ static eas_status launch_kernel(void (*kern)(Params), int grid, int block, size_
   cfg.stream = stream;
   cudaLaunchAttribute attr[2];
   int n = 0;
-  attr[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  attr[n].val.programmaticStreamSerializationAllowed = 1;
-  ++n;
+  if (g_overlap_launches) {
+    attr[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[n].val.programmaticStreamSerializationAllowed = 1;
+    ++n;
+  }
   if (cluster > 1) {
     attr[n].id = cudaLaunchAttributeClusterDimension;
     attr[n].val.clusterDim.x = static_cast<unsigned>(cluster);
@@ -627,6 +654,7 @@ struct GemmCall {
   const float2* rope_cs = nullptr;
   int reverse = 0;             // walk the tiles last to first
   int w_const = 1;             // the weights are constant (set at create time): their loads may start before the stream's earlier work ends
+  int force_tile = 0;          // 0: the launcher picks; 1 one CTA per 128x256 tile, 2 CTA pair per 256x256, 3 pair per 256x512 (tests)
   int splits = 1;              // split K (see GemmParams::splits); the partial sums of splits 1.. go to `part`
   float* part = nullptr;       // [(splits - 1) * part_rows, N] fp32
   int64_t part_rows = 0;
@@ -664,6 +692,12 @@ static eas_status launch_gemm(const GemmCall& g, int budget, cudaStream_t stream
     if (tma_out && g.act != ACT_SWIGLU && k_total >= 2048 && L.N % 512 == 0 && gemm_kernel_for(g.act, g.out_fp32, 3) != nullptr) {
       const double cost_wide = waves(m256 * (L.N / (2 * kBN)) * g.splits, pairs) * (kb / g.splits * 0.75 + 4.0);
       if (cost_wide < std::min(cost_single, cost_pair)) { ctas = 2; wide = true; }
+    }
+    if (g.force_tile != 0) {
+      const bool wide_ok = tma_out && g.act != ACT_SWIGLU && L.N % 512 == 0 && gemm_kernel_for(g.act, g.out_fp32, 3) != nullptr;
+      if (g.force_tile == 3 && !wide_ok) return fail(EAS_ERR_UNSUPPORTED, "no wide (256x512) tile for this GEMM: it needs N %% 512 == 0, a plain or GELU epilogue and row-aligned output");
+      ctas = g.force_tile == 1 ? 1 : 2;
+      wide = g.force_tile == 3;
     }
 #ifdef EAS_GEMM_FORCE_TILE   // calibration builds only: 1 single CTA, 2 pair, 3 wide pair (where a wide kernel exists)
     ctas = EAS_GEMM_FORCE_TILE == 1 ? 1 : 2;
@@ -723,6 +757,7 @@ static eas_status launch_norm_nv(const NormParams& p, int budget, cudaStream_t s
     static OncePerDevice once;                                                                                     \
     if (once.first()) {                                                                                            \
       CUDA_TRY(cudaFuncSetAttribute(norm_kernel<NV_, KIND, F32, PART>, cudaFuncAttributeMaxDynamicSharedMemorySize, kOnePerSmSmem)); \
+      once.settled();                                                                                              \
     }                                                                                                              \
     EAS_TRY(launch_kernel(norm_kernel<NV_, KIND, F32, PART>, std::min(budget, (p.rows + 15) / 16), 512, kOnePerSmSmem, stream, p)); \
     break;                                                                                                         \
@@ -748,7 +783,7 @@ static eas_status launch_norm(int kind, bool out_fp32, const NormParams& p, int 
   }
   if (kind == NORM_LN) return out_fp32 ? launch_norm_nv<NORM_LN, true>(p, budget, stream) : launch_norm_nv<NORM_LN, false>(p, budget, stream);
   if (kind == NORM_RMS) return out_fp32 ? launch_norm_nv<NORM_RMS, true>(p, budget, stream) : launch_norm_nv<NORM_RMS, false>(p, budget, stream);
-  if (kind == NORM_CAST) return out_fp32 ? fail(EAS_ERR_UNSUPPORTED, "fp32 cast") : launch_norm_nv<NORM_CAST, false>(p, budget, stream);
+  if (kind == NORM_CAST) return out_fp32 ? launch_norm_nv<NORM_CAST, true>(p, budget, stream) : launch_norm_nv<NORM_CAST, false>(p, budget, stream);
   return fail(EAS_ERR_INVALID_ARG, "unknown norm kind %d", kind);
 }
 
@@ -792,6 +827,7 @@ static eas_status launch_attention_mma(const bf16* qkv, bf16* out, const int32_t
   if (once.first()) {
     CUDA_TRY(cudaFuncSetAttribute(attn_mma_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, kOnePerSmSmem));
     CUDA_TRY(cudaFuncSetAttribute(attn_mma_kernel<80>, cudaFuncAttributeMaxDynamicSharedMemorySize, kOnePerSmSmem));
+    once.settled();
   }
   static_assert(attn_mma_smem_bytes<80>() <= kOnePerSmSmem, "attention tile does not fit");
   if (hd == 64) return launch_kernel(attn_mma_kernel<64>, grid, kAttnThreads, kOnePerSmSmem, stream, ap);
@@ -840,6 +876,7 @@ static eas_status launch_attention_tc(const bf16* qkv, bf16* out, const int32_t*
     CUDA_TRY(cudaFuncSetAttribute(attn_tc_kernel<80, PT>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttnTcSmem<80, PT>::kBytes));
     if (AttnTcSmem<64, PT>::kDualHeadOk)
       CUDA_TRY(cudaFuncSetAttribute(attn_tc_kernel<64, PT, AttnTcSmem<64, PT>::kDualHeadOk>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttnTcSmem<64, PT>::kBytes));
+    once.settled();
   }
   if (hd == 64 && dual)
     return launch_kernel(attn_tc_kernel<64, PT, AttnTcSmem<64, PT>::kDualHeadOk>, grid, kTcThreads, AttnTcSmem<64, PT>::kBytes, stream, ap);
@@ -864,6 +901,13 @@ static eas_status encode_impl(eas_encoder* e, const eas_packed_inputs* in, void*
   if (in->data == nullptr || in->item_shape == nullptr || in->item_offset == nullptr || in->cu_seqlens_host == nullptr ||
       workspace == nullptr || cu_dev == nullptr || out_embeddings == nullptr)
     return fail(EAS_ERR_INVALID_ARG, "a required pointer is null");
+  {
+    // the handle's weights, tensor maps and kernel attributes belong to the device it was created on
+    int dev = -1;
+    CUDA_TRY(cudaGetDevice(&dev));
+    if (dev != e->device)
+      return fail(EAS_ERR_INVALID_ARG, "the encoder was created on device %d but device %d is current", e->device, dev);
+  }
   const int n = in->n_items;
   if (n < 1 || n > EAS_MAX_ITEMS) return fail(EAS_ERR_INVALID_ARG, "n_items %d outside 1..%d", n, static_cast<int>(EAS_MAX_ITEMS));
   if (sm_budget < 0 || sm_budget > e->sm_count) return fail(EAS_ERR_INVALID_ARG, "sm_budget %d outside 0..%d", sm_budget, e->sm_count);
@@ -871,6 +915,7 @@ static eas_status encode_impl(eas_encoder* e, const eas_packed_inputs* in, void*
   if ((reinterpret_cast<uintptr_t>(in->data) & 15) != 0 || (reinterpret_cast<uintptr_t>(out_embeddings) & 15) != 0)
     return fail(EAS_ERR_INVALID_ARG, "data / out_embeddings must be 16-byte aligned");
   const int budget = sm_budget == 0 ? e->sm_count : sm_budget;
+  g_overlap_launches = budget == e->sm_count;
   const eas_arch_config& c = e->cfg;
   const int32_t* cu = in->cu_seqlens_host;
   const int d = c.d_model;
@@ -892,10 +937,11 @@ static eas_status encode_impl(eas_encoder* e, const eas_packed_inputs* in, void*
     items.offset[i] = in->item_offset[i];
     if (audio) {
       if (h != c.in_channels || w != 1) return fail(EAS_ERR_INVALID_ARG, "audio item %d must be (frames, %d, 1)", i, c.in_channels);
-      if (f % 2 != 0) return fail(EAS_ERR_INVALID_ARG, "audio item %d has an odd frame count", i);
       if ((in->item_offset[i] * 2) % 16 != 0) return fail(EAS_ERR_INVALID_ARG, "item %d offset is not 16-byte aligned", i);
-      expect = f / 2;
-      aux += f + 2;
+      // the stride-2 convolution (k = 3, padding 1) yields ceil(f / 2) tokens; the staging rows of an item are one zero
+      // row, its f frames, and one zero row (two when f is odd, so that every item starts on an even staging row)
+      expect = (f + 1) / 2;
+      aux += f + 2 + (f & 1);
     } else {
       const int unit = c.patch * (c.head == EAS_HEAD_MERGER_2X2 ? 2 : 1);
       if (h % unit != 0 || w % unit != 0) return fail(EAS_ERR_INVALID_ARG, "item %d: height/width must be multiples of %d", i, unit);
@@ -963,7 +1009,10 @@ static eas_status encode_impl(eas_encoder* e, const eas_packed_inputs* in, void*
     sp.data = static_cast<const bf16*>(in->data); sp.mel_pad = mel_pad; sp.h1_pad = h1_pad;
     sp.n_mel = c.in_channels; sp.d_model = d; sp.padded_rows = static_cast<int>(pl.padded_rows); sp.items = items;
     static OncePerDevice once;
-    if (once.first()) CUDA_TRY(cudaFuncSetAttribute(audio_stage_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kOnePerSmSmem));
+    if (once.first()) {
+      CUDA_TRY(cudaFuncSetAttribute(audio_stage_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kOnePerSmSmem));
+      once.settled();
+    }
     EAS_TRY(mark(e, EAS_KC_EMBED_GATHER, stream));
     EAS_TRY(launch_kernel(audio_stage_kernel, budget, 512, kOnePerSmSmem, stream, sp));
     ++launches;
@@ -987,7 +1036,10 @@ static eas_status encode_impl(eas_encoder* e, const eas_packed_inputs* in, void*
     ip.merge_order = c.family == EAS_FAMILY_VIT_ROPE_MERGER ? 1 : 0;
     ip.items = items;
     static OncePerDevice once;
-    if (once.first()) CUDA_TRY(cudaFuncSetAttribute(im2col_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kOnePerSmSmem));
+    if (once.first()) {
+      CUDA_TRY(cudaFuncSetAttribute(im2col_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kOnePerSmSmem));
+      once.settled();
+    }
     EAS_TRY(mark(e, EAS_KC_EMBED_GATHER, stream));
     EAS_TRY(launch_kernel(im2col_kernel, budget, 512, kOnePerSmSmem, stream, ip));
     ++launches;
@@ -1069,13 +1121,14 @@ static eas_status encode_impl(eas_encoder* e, const eas_packed_inputs* in, void*
 
   // ---- connector
   EAS_TRY(mark(e, EAS_KC_NORM, stream));
+  const bool out_f32 = c.out_dtype == EAS_OUT_FP32;
   if (c.head == EAS_HEAD_NONE) {
     if (c.final_norm) {
       NormParams np{x, out_embeddings, e->fng, e->fnb, nullptr, static_cast<int>(T), d, c.norm_eps};
-      EAS_TRY(launch_norm(ln_kind, false, np, budget, stream)); ++launches;
+      EAS_TRY(launch_norm(ln_kind, out_f32, np, budget, stream)); ++launches;
     } else {
       NormParams np{x, out_embeddings, nullptr, nullptr, nullptr, static_cast<int>(T), d, c.norm_eps};
-      EAS_TRY(launch_norm(NORM_CAST, false, np, budget, stream)); ++launches;
+      EAS_TRY(launch_norm(NORM_CAST, out_f32, np, budget, stream)); ++launches;
     }
   } else {
     int64_t rows_in;   // rows of the connector's first GEMM
@@ -1097,7 +1150,7 @@ static eas_status encode_impl(eas_encoder* e, const eas_packed_inputs* in, void*
     EAS_TRY(launch_gemm(g1, budget, stream, status)); ++launches;
     GemmCall g2;
     g2.A = abuf; g2.a_run = c.d_head_hidden; g2.a_row_elems = c.d_head_hidden; g2.a_rows = rows_in; g2.M = static_cast<int>(rows_in); g2.lin = &e->head2;
-    g2.out = out_embeddings; g2.ldo = c.d_out;
+    g2.out = out_embeddings; g2.ldo = c.d_out; g2.out_fp32 = out_f32 ? 1 : 0;
     EAS_TRY(mark(e, EAS_KC_GEMM_HEAD, stream));
     EAS_TRY(launch_gemm(g2, budget, stream, status)); ++launches;
   }
@@ -1223,6 +1276,8 @@ extern "C" eas_status eas_encode_microbatch_static(eas_encoder* e, const eas_pac
   int dev = 0;
   CUDA_TRY(cudaGetDevice(&dev));
   if (dev < 0 || dev >= kMaxDevices) return fail(EAS_ERR_UNSUPPORTED, "device ordinal %d", dev);
+  if (e != nullptr && dev != e->device)
+    return fail(EAS_ERR_INVALID_ARG, "the encoder was created on device %d but device %d is current", e->device, dev);
   unsigned char* base = nullptr;
   {
     std::lock_guard<std::mutex> lock(g_static_mutex);
@@ -1381,20 +1436,27 @@ static eas_status resolve_budget(int32_t sm_budget, int* budget) {
   EAS_TRY(device_check(&sm_count));
   if (sm_budget < 0 || sm_budget > sm_count) return fail(EAS_ERR_INVALID_ARG, "sm_budget %d outside 0..%d", sm_budget, sm_count);
   *budget = sm_budget == 0 ? sm_count : sm_budget;
+  g_overlap_launches = *budget == sm_count;
   return EAS_OK;
 }
 
 extern "C" eas_status eas_kernel_gemm(const void* A, const void* W, const void* bias, void* out, const float* resid,
                                       int32_t M, int32_t N, int32_t K, int32_t act, int32_t out_fp32, int32_t sm_budget,
                                       void* stream, uint32_t* status_dev) {
+  return eas_kernel_gemm_tile(A, W, bias, out, resid, M, N, K, act, out_fp32, sm_budget, stream, status_dev, 0);
+}
+
+extern "C" eas_status eas_kernel_gemm_tile(const void* A, const void* W, const void* bias, void* out, const float* resid,
+                                           int32_t M, int32_t N, int32_t K, int32_t act, int32_t out_fp32, int32_t sm_budget,
+                                           void* stream, uint32_t* status_dev, int32_t tile_shape) {
+  if (tile_shape < 0 || tile_shape > 3) return fail(EAS_ERR_INVALID_ARG, "tile_shape %d outside 0..3", tile_shape);
   if (A == nullptr || W == nullptr || bias == nullptr || out == nullptr || status_dev == nullptr)
     return fail(EAS_ERR_INVALID_ARG, "a required pointer is null");
   if (M <= 0 || N <= 0 || K <= 0 || K % 64 != 0 || N % 32 != 0) return fail(EAS_ERR_INVALID_ARG, "need M,N,K > 0, K %% 64 == 0, N %% 32 == 0");
   if (act < 0 || act > 2 || (act == ACT_SWIGLU && out_fp32)) return fail(EAS_ERR_INVALID_ARG, "bad epilogue selection");
   int budget = 0;
   EAS_TRY(resolve_budget(sm_budget, &budget));
-  static OncePerDevice once;
-  if (once.first()) EAS_TRY(set_kernel_attributes());
+  EAS_TRY(set_kernel_attributes_once());
   Linear L;
   L.w = static_cast<const bf16*>(W); L.b = static_cast<const bf16*>(bias); L.N = N; L.K = K;
   EAS_TRY(finish_linear(L));
@@ -1402,6 +1464,7 @@ extern "C" eas_status eas_kernel_gemm(const void* A, const void* W, const void* 
   g.A = A; g.a_run = K; g.a_row_elems = K; g.a_rows = M; g.M = M; g.lin = &L; g.act = act; g.out_fp32 = out_fp32;
   g.out = out; g.ldo = act == ACT_SWIGLU ? N / 2 : N; g.resid = out_fp32 ? resid : nullptr;
   g.w_const = 0;             // W is the caller's tensor: work earlier in the stream may have produced it
+  g.force_tile = budget >= 2 ? tile_shape : 0;
   return launch_gemm(g, budget, static_cast<cudaStream_t>(stream), status_dev);
 }
 

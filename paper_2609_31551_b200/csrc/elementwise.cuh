@@ -282,7 +282,7 @@ __global__ void __launch_bounds__(256) prep_kernel(const __grid_constant__ PrepP
       const int t = m - p.items.aux_start[it];
       p.conv1_row_map[m] = t < p.items.frames[it] ? m + 1 : -1;
     }
-    // conv2 walks (frames/2 + 1) rows per item; the last one is dropped
+    // conv2 walks (ceil(frames/2) + 1) rows per item; the last one is dropped
     for (int m = gtid; m < p.n_embed_rows; m += gsz) {
       // aux_start[i] / 2 is the conv2 row prefix because every padded item has an even row count
       int lo = 0, hi = n - 1;
@@ -291,15 +291,15 @@ __global__ void __launch_bounds__(256) prep_kernel(const __grid_constant__ PrepP
         if ((p.items.aux_start[mid] >> 1) <= m) lo = mid; else hi = mid - 1;
       }
       const int t = m - (p.items.aux_start[lo] >> 1);
-      const bool ok = t < (p.items.frames[lo] >> 1);
+      const bool ok = t < ((p.items.frames[lo] + 1) >> 1);
       p.embed_row_map[m] = ok ? p.items.tok_start[lo] + t : -1;
       p.embed_pos_idx[m] = ok ? t : 0;
     }
   }
 }
 
-// audio: copy mel frames into a staging buffer with one zero row before and after each item, and
-// zero the matching pad rows of the h1 staging buffer
+// audio: copy mel frames into a staging buffer with one zero row before and one (odd frame counts: two) after each
+// item, and zero the matching pad rows of the h1 staging buffer
 struct AudioStageParams {
   const bf16* data;
   bf16* mel_pad;       // [padded rows, n_mel]
@@ -322,12 +322,14 @@ __global__ void __launch_bounds__(512, 1) audio_stage_kernel(const __grid_consta
     if (t >= 0 && t < p.items.frames[it]) v = p.data[p.items.offset[it] + static_cast<long long>(t) * p.n_mel + c];
     p.mel_pad[idx] = v;
   }
-  const long long pad_total = static_cast<long long>(p.items.n_items) * 2 * p.d_model;
+  // pad rows of h1: the item's first staging row and every row behind its last frame (one, or two for an odd count)
+  const long long pad_total = static_cast<long long>(p.items.n_items) * 3 * p.d_model;
   for (long long idx = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x; idx < pad_total; idx += gsz) {
     const int c = static_cast<int>(idx % p.d_model);
     const int which = static_cast<int>(idx / p.d_model);
-    const int it = which >> 1;
-    const int row = (which & 1) ? p.items.aux_start[it + 1] - 1 : p.items.aux_start[it];
+    const int it = which / 3, k = which - it * 3;
+    const int row = k == 0 ? p.items.aux_start[it] : p.items.aux_start[it + 1] - k;
+    if (k == 2 && (p.items.frames[it] & 1) == 0) continue;      // even count: that row holds the last frame
     p.h1_pad[static_cast<long long>(row) * p.d_model + c] = __float2bfloat16(0.f);
   }
 }

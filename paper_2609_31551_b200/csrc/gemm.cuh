@@ -130,6 +130,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_kernel(const __grid_cons
   uint64_t* acc_full = bars + 2 * kMaxStages;      // [2]        MMA -> epilogue (pair: signalled in both CTAs)
   uint64_t* acc_empty = bars + 2 * kMaxStages + 2; // [2]        epilogue -> MMA (pair: both CTAs' warps arrive at the leader)
   uint64_t* bias_bar = bars + 2 * kMaxStages + 4;  // [2]        epilogue warps: bias values staged
+  uint64_t* bias_free = bars + 2 * kMaxStages + 7; // [1]        wide tiles: every epilogue warp has read the staged bias
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kMaxStages + 6);
   volatile uint32_t* abort_flag = tmem_slot + 1;
 
@@ -147,6 +148,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_kernel(const __grid_cons
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
     for (int a = 0; a < 2; ++a) { mbar_init(&acc_full[a], 1); mbar_init(&acc_empty[a], kEpiWarps * CTAS); mbar_init(&bias_bar[a], kEpiWarps); }
+    mbar_init(bias_free, kEpiWarps);
     *abort_flag = 0;
     mbar_fence_init();
     tma_prefetch_desc(&p.tma_a);
@@ -187,6 +189,10 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_kernel(const __grid_cons
         for (int kb = kb0; kb < kb1; ++kb, ++it) {
           const int s = it % kStages;
           const uint32_t ph = (it / kStages) & 1u;
+          // The W producer of constant weights skipped the grid-dependency wait above and has filled every stage once;
+          // its next wait needs the consumer, which needs A, which needs the earlier kernels: join the dependency first,
+          // so that the bounded wait below never runs while a predecessor is still working.
+          if (do_b && p.w_const && it == kStages) pdl_wait();
           if (!mbar_wait(&empty_bar[s], ph ^ 1u, abort_flag)) { ok = false; break; }
           uint8_t* sa = smem + s * kStageBytes;
           uint8_t* sb = sa + kABytes * KD;
@@ -304,6 +310,10 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_kernel(const __grid_cons
         // ---- staged path: bias from shared memory, 32-row sub-tiles written to a swizzled staging buffer
         //      and stored (or reduce-added, for the fp32 residual stream) by TMA; rows >= M are clipped by TMA
         float* sbias = reinterpret_cast<float*>(smem + kBiasOff) + acc * 256;   // wide tiles use both halves as one
+        // With two accumulator buffers the other buffer's bias_bar (eight arrivals) lies between two uses of a bias slot
+        // and orders them.  A wide tile has ONE slot: nobody may overwrite it before all eight warps have finished
+        // reading the previous tile's values (each arrives at bias_free after its last chunk).
+        if (kAccBuffers == 1 && tcount > 0 && !mbar_wait(bias_free, (tcount - 1) & 1u, abort_flag)) { ok = false; break; }
         {
 #pragma unroll
           for (int h = 0; h < NW; ++h) {
@@ -464,6 +474,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_kernel(const __grid_cons
         }
         }
         release_accumulator(acc);
+        if (kAccBuffers == 1 && lane == 0) mbar_arrive(bias_free);   // this warp's reads of the staged bias are done (after the __syncwarp above)
         GEMM_STAMP(11);
         if (tcount == 0 && ew == 0 && lane == 0) GEMM_TL(5);
         continue;

@@ -73,6 +73,46 @@ def test_gemm_is_independent_of_sm_budget(N, K):
         assert torch.equal(out, ref), budget
 
 
+@pytest.mark.parametrize("act,out_fp32", [(0, False), (1, False), (0, True)])
+def test_gemm_tile_shapes_agree_bit_for_bit_with_large_distinct_biases(act, out_fp32):
+    """The three tile shapes must give the same bits.  The bias is large and different in every 512-column block, the
+    budget is small so that every CTA (pair) walks many tiles back to back, and the whole thing is repeated: a tile
+    that picked up its neighbour's staged bias (the wide tile has a single bias slot that the next tile overwrites)
+    would differ from the other shapes by whole units."""
+    import paper_2609_31551_b200 as P
+    rng = np.random.Generator(np.random.PCG64(91))
+    M, N, K = 1300, 2048, 2048
+    A, W = _dev(_bf16_exact(rng, (M, K))), _dev(_bf16_exact(rng, (N, K), 0.02))
+    bias = np.repeat(np.arange(N // 256, dtype=np.float32) * 8.0 - 24.0, 256) + rng.standard_normal(N).astype(np.float32)
+    b = _dev(S.round_to_bf16(bias))
+    resid = torch.from_numpy(rng.standard_normal((M, N)).astype(np.float32)).cuda() if out_fp32 else None
+    ref, st = P.kernel_gemm(A, W, b, act=act, out_fp32=out_fp32, resid=resid, sm_budget=2, tile_shape=1)
+    torch.cuda.synchronize()
+    assert int(st[0]) == 0
+    y = O.linear(O._t(A.float().cpu().numpy()), O._t(W.float().cpu().numpy()), O._t(b.float().cpu().numpy()))
+    if act == 1:
+        y = O.gelu(y)
+    if out_fp32:
+        y = y + resid.double().cpu()
+    assert (ref.double().cpu() - y).abs().max() <= 2.0 ** -7 * float(y.abs().max())
+    for shape in (2, 3):
+        for budget in (2, 6, 148):
+            for _ in range(3):
+                out, st = P.kernel_gemm(A, W, b, act=act, out_fp32=out_fp32, resid=resid, sm_budget=budget, tile_shape=shape)
+                torch.cuda.synchronize()
+                assert int(st[0]) == 0
+                assert torch.equal(out, ref), (shape, budget)
+
+
+def test_gemm_wide_tile_is_refused_where_it_does_not_exist():
+    import paper_2609_31551_b200 as P
+    rng = np.random.Generator(np.random.PCG64(92))
+    A, W, b = _dev(_bf16_exact(rng, (300, 256))), _dev(_bf16_exact(rng, (768, 256), 0.05)), _dev(_bf16_exact(rng, (768,)))
+    with pytest.raises(P.EasError) as e:
+        P.kernel_gemm(A, W, b, tile_shape=3)         # N = 768 is not a multiple of 512
+    assert e.value.status == 2
+
+
 @pytest.mark.parametrize("d", [256, 1024, 1280])
 @pytest.mark.parametrize("kind", [0, 1, 2])
 def test_norm(d, kind):

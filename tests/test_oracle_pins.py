@@ -190,14 +190,14 @@ def test_sinusoid_table():
 
 def _tiny_cfg(family):
     if family == 0:
-        return dict(name="t0", family=0, n_layers=1, d_model=8, n_heads=2, d_mlp=12, norm=0, norm_eps=1e-5, mlp=0,
+        return dict(name="t0", family=0, n_layers=2, d_model=8, n_heads=2, d_mlp=12, norm=0, norm_eps=1e-5, mlp=0,
                     in_channels=2, patch=2, temporal_patch=1, has_cls=1, embed_norm=1, final_norm=1, pos=0,
                     max_pos=9, rope_theta=0.0, head=1, d_head_hidden=6, d_out=5)
     if family == 1:
-        return dict(name="t1", family=1, n_layers=1, d_model=16, n_heads=2, d_mlp=12, norm=1, norm_eps=1e-6, mlp=1,
+        return dict(name="t1", family=1, n_layers=2, d_model=16, n_heads=2, d_mlp=12, norm=1, norm_eps=1e-6, mlp=1,
                     in_channels=2, patch=2, temporal_patch=2, has_cls=0, embed_norm=0, final_norm=0, pos=1,
                     max_pos=0, rope_theta=100.0, head=2, d_head_hidden=10, d_out=6)
-    return dict(name="t2", family=2, n_layers=1, d_model=8, n_heads=2, d_mlp=12, norm=0, norm_eps=1e-5, mlp=0,
+    return dict(name="t2", family=2, n_layers=2, d_model=8, n_heads=2, d_mlp=12, norm=0, norm_eps=1e-5, mlp=0,
                 in_channels=3, patch=1, temporal_patch=1, has_cls=0, embed_norm=0, final_norm=1, pos=0,
                 max_pos=8, rope_theta=0.0, head=0, d_head_hidden=0, d_out=8)
 
@@ -225,6 +225,41 @@ def test_tiny_encoder_against_pure_python_brute_force(family):
         assert got.shape == ref.shape
         assert np.abs(got - ref).max() < 1e-11 * max(1.0, np.abs(ref).max())
         assert np.abs(ref).max() > 1e-3
+
+
+@pytest.mark.parametrize("family", [0, 1, 2])
+def test_layer_loop_reads_each_layers_own_weights(family):
+    """Two layers with different weights: exchanging blk0.* and blk1.* must change the output (a loop that read one
+    layer's weights twice, or the layers in the wrong order, would not notice), and exchanging twice restores it.
+    The brute-force test above pins the right order; this one pins that the order matters at all."""
+    cfg = _tiny_cfg(family)
+    assert cfg["n_layers"] == 2
+    w = S.make_weights(cfg, seed=31 + family, profile="sharp")
+    w = {k: (v * 10 if k.endswith(".w") else v).astype(np.float64) for k, v in w.items()}
+    swapped = {}
+    for k, v in w.items():
+        if k.startswith("blk0."):
+            swapped["blk1." + k[5:]] = v
+        elif k.startswith("blk1."):
+            swapped["blk0." + k[5:]] = v
+        else:
+            swapped[k] = v
+    assert any(not np.array_equal(w[k], swapped[k]) for k in w if k.startswith("blk"))
+    item = _tiny_items(cfg, 21)[1]
+    a = O.encode_item(cfg, w, item).numpy()
+    b = O.encode_item(cfg, swapped, item).numpy()
+    assert np.abs(a - b).max() > 1e-3 * np.abs(a).max()
+    # the taps after block 0 must already differ (block 0 reads blk0.*, not blk1.*)
+    ta, tb = {}, {}
+    O.encode_item(cfg, w, item, taps=ta)
+    O.encode_item(cfg, swapped, item, taps=tb)
+    assert (ta["blk0"] - tb["blk0"]).abs().max() > 1e-6
+    # one layer of the swapped weights == running only blk1 of the original: block 0 of `swapped` IS blk1 of `w`
+    cfg1 = dict(cfg, n_layers=1)
+    w_only1 = {k: v for k, v in swapped.items() if not k.startswith("blk1.")}
+    t1 = {}
+    O.encode_item(cfg1, w_only1, item, taps=t1)
+    assert torch.equal(t1["blk0"], tb["blk0"])
 
 
 @pytest.mark.parametrize("family", [0, 1, 2])
@@ -289,7 +324,7 @@ def test_merger_is_gather_over_2x2_neighbourhoods():
     clip = np.random.Generator(np.random.PCG64(2)).random((2, 2, 8, 12))   # gt=1, gh=4, gw=6
     taps = {}
     out = O.encode_item(cfg, w, clip, taps=taps).numpy()
-    x = taps["blk0"]
+    x = taps[f"blk{cfg['n_layers'] - 1}"]          # residual stream after the last block
     n = O.rms_norm(x, O._t(w["head.norm.g"]), cfg["norm_eps"])
     _, hpos, wpos = O.merge_order_positions(1, 4, 6)
     index_of = {(int(h), int(c)): i for i, (h, c) in enumerate(zip(hpos, wpos))}

@@ -1,43 +1,56 @@
-"""The allocation-free entry point (eas_encode_microbatch_static) against the ordinary one.
+"""The allocation-free entry point (eas_encode_microbatch_static) against the ordinary one and the oracle.
 
 Some callers of the encoder cannot allocate device memory: a worker that shares its GPU with a neighbour
 that already owns the rest of HBM, or a serving loop where an allocation may stall the device.  For them the
-library carries its own scratch array.  This test calls that entry point through the C ABI twice in a row (the
-array keeps the first call's contents, so the second call shows that nothing stale is read) and compares both
-results with eas_encode_microbatch on a caller-allocated workspace.  It also checks that a micro-batch too large
-for the built-in scratch is refused with a clear error.  Collected last on purpose."""
+library carries its own scratch array.  These tests call that entry point through the C ABI twice in a row (the
+array keeps the first call's contents, so the second call shows that nothing stale is read).  Both entry points
+run the same kernels in the same order, so their results must be the same BYTES, not merely close; and each
+result is also held against the CPU oracle with the tolerance of the other parity tests.  One case per encoder
+family, so that every scratch region (patch operand, row maps, rotary table, padded mel / convolution rows) is
+covered.  A micro-batch too large for the built-in scratch must be refused with a clear error.
+Collected last on purpose."""
 import numpy as np
 import pytest
 import torch
 
 import eas_synth as S
+from oracle import encoder_oracle as O
 from tests import gpu_util as G
 
 pytestmark = pytest.mark.gpu
 
+CASES = {
+    # family: (config, overrides, [first micro-batch, second micro-batch])
+    "vit_table": ("c0", {}, [[(1, 224, 224)] * 3, [(1, 224, 224)] * 2]),
+    "vit_rope_merger": ("c2", dict(n_layers=2), [[(1, 224, 224), (1, 56, 84)], [(1, 28, 28), (1, 140, 364), (1, 56, 56)]]),
+    "audio_conv": ("c4", dict(n_layers=1), [[(200, 128, 1), (7, 128, 1)], [(2, 128, 1), (600, 128, 1), (64, 128, 1)]]),
+}
 
-def test_static_scratch_entry_point_matches_and_repeats():
+
+@pytest.mark.parametrize("family", list(CASES))
+def test_static_scratch_entry_point_matches_and_repeats(family):
     import paper_2609_31551_b200 as P
-    cfg = S.get_config("c0")
+    name, over, batches = CASES[family]
+    cfg = S.get_config(name, **over)
     w = S.make_weights(cfg)
     enc = P.Encoder(cfg, P.weights_to_device(w))
-    outs = []
-    for seed, n in ((11, 3), (12, 2)):            # two different micro-batches, back to back
-        shapes = [(1, 224, 224)] * n
-        items = S.make_items(cfg, shapes, seed=seed)
+    runs = []
+    for k, shapes in enumerate(batches):            # two different micro-batches, back to back on the same scratch
+        items = S.make_items(cfg, shapes, seed=11 + k)
         data, offsets = P.pack_items(items)
         cu = G.cu_seqlens_of(cfg, items)
         cu_dev = torch.from_numpy(cu).cuda()
-        ref = enc.encode_microbatch(data, shapes, offsets, cu, cu_seqlens_dev=cu_dev)
+        assert enc.workspace_bytes(int(cu[-1]), len(shapes)) < (32 << 20) - 1024
+        want = enc.encode_microbatch(data, shapes, offsets, cu, cu_seqlens_dev=cu_dev)
         enc.status()
-        out = torch.zeros_like(ref)
+        out = torch.full_like(want, float("nan"))
         enc.encode_microbatch_static(data, shapes, offsets, cu, cu_dev, out)
         enc.status()
-        outs.append((out, ref))
-    for out, ref in outs:
-        got, want = out.double().cpu().numpy(), ref.double().cpu().numpy()
-        assert np.isfinite(got).all()
-        G.assert_parity(got, want, "static-scratch entry point vs workspace entry point")
+        runs.append((items, out, want))
+    for items, out, want in runs:
+        assert torch.equal(out, want), "static-scratch entry point differs from the workspace entry point"
+        ref, _, _ = O.encode_microbatch(cfg, w, items)
+        G.assert_parity(out.double().cpu().numpy(), ref, f"static-scratch entry point vs oracle ({family})")
 
 
 def test_static_scratch_rejects_a_micro_batch_that_does_not_fit():
