@@ -28,112 +28,31 @@ sys.path.insert(0, ROOT)
 import eas_synth as S  # noqa: E402
 
 
-# ------------------------------------------------------------------ algorithmic work (real tokens only)
-def flops_of(cfg, shapes):
-    """Algorithmic FLOPs of one forward pass: 2*M*N*K per linear map, 4*d*S^2 per item and layer for attention."""
-    d, I, L = cfg["d_model"], cfg["d_mlp"], cfg["n_layers"]
-    seqs = [S.tokens_per_item(cfg, s) for s in shapes]
-    T = sum(seqs)
-    mlp = (6 if cfg["mlp"] == 1 else 4) * d * I
-    lin = L * T * (8 * d * d + mlp)
-    attn = L * 4 * d * sum(s * s for s in seqs)
-    if cfg["family"] == 2:
-        emb = sum(2 * s[0] * 3 * cfg["in_channels"] * d + 2 * (s[0] // 2) * 3 * d * d for s in shapes)
-    else:
-        emb = 2 * (T - (len(shapes) if cfg["has_cls"] else 0)) * S.configs.embed_k(cfg) * d
-    head = 0
-    out_rows = sum(S.out_tokens_per_item(cfg, s) for s in shapes)
-    if cfg["head"] == 1:
-        head = 2 * out_rows * (d * cfg["d_head_hidden"] + cfg["d_head_hidden"] * cfg["d_out"])
-    elif cfg["head"] == 2:
-        head = 2 * out_rows * (4 * d * cfg["d_head_hidden"] + cfg["d_head_hidden"] * cfg["d_out"])
-    return dict(total=lin + attn + emb + head, linear=lin + emb + head, attention=attn, tokens=T, out_rows=out_rows,
-                sum_s2=sum(s * s for s in seqs))
+from paper_2609_31551_b200.measure import (ClockSampler, Point, flops_of, gemm_flops_by_class, measured_peaks,  # noqa: E402
+                                           time_point, workload)
 
-
-def gemm_flops_by_class(cfg, shapes):
-    """Algorithmic FLOPs per kernel class of the GEMMs (keys = EAS_KC_* ids)."""
-    d, I, L = cfg["d_model"], cfg["d_mlp"], cfg["n_layers"]
-    f = flops_of(cfg, shapes)
-    T = f["tokens"]
-    up = (4 if cfg["mlp"] == 1 else 2) * d * I
-    emb = f["linear"] - L * T * (8 * d * d + (6 if cfg["mlp"] == 1 else 4) * d * I)
-    head = 0
-    if cfg["head"]:
-        kin = 4 * d if cfg["head"] == 2 else d
-        head = 2 * f["out_rows"] * (kin * cfg["d_head_hidden"] + cfg["d_head_hidden"] * cfg["d_out"])
-    return {2: emb - head, 4: L * T * 6 * d * d, 6: L * T * 2 * d * d, 7: L * T * up, 8: L * T * 2 * d * I, 9: head,
-            5: f["attention"]}
-
-
-class ClockSampler:
-    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
-    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
-         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
-
-    def __init__(self, gpu_index: int):
-        self.gpu = gpu_index
-        self.proc = None
-        self.lines = []
-
-    def start(self):
-        try:
-            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.gpu}", f"--query-gpu={self.Q}",
-                                          "--format=csv,noheader,nounits", "-lms", "100"],
-                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
-            self.thread = threading.Thread(target=self._read, daemon=True)
-            self.thread.start()
-        except Exception:
-            self.proc = None
-
-    def _read(self):
-        for line in self.proc.stdout:
-            self.lines.append(line.strip())
-
-    def stop(self):
-        if self.proc is None:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
-        self.proc.terminate()
-        try:
-            self.proc.wait(timeout=5)
-        except Exception:
-            self.proc.kill()
-        sm, mx, reasons, pw = [], [], set(), []
-        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for ln in self.lines:
-            parts = [p.strip() for p in ln.split(",")]
-            if len(parts) < 7:
-                continue
-            try:
-                sm.append(float(parts[0])); mx.append(float(parts[1])); pw.append(float(parts[2]))
-            except ValueError:
-                continue
-            for nm, val in zip(names, parts[3:7]):
-                if val.lower().startswith("active"):
-                    reasons.add(nm)
-        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "power_w_max": max(pw) if pw else None, "samples": len(sm), "reasons": sorted(reasons)}
-
-
-def measured_peaks():
-    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
-    if os.path.exists(path):
-        with open(path) as f:
-            p = json.load(f)
-        return dict(hbm=p["hbm_gbs"], burst=p["bf16_tflops"], sustained=p["bf16_tflops_sustained"], source="measured")
-    return dict(hbm=6650.0, burst=1590.0, sustained=1400.0, source="fallback")
+# The points of the headline metric (tokens/s and items/s against micro-batch and sm_budget) that the default run
+# measures besides the main one, grouped by configuration so that every encoder is built once:
+# (config, [(micro-batch, [sm budgets])]).  0 = all SMs.
+SWEEP = [
+    ("c1", [(1, [0]), (16, [0]), (64, [0]), (32, [37, 74, 111])]),
+    ("c3", [(1, [0, 37, 74, 111]), (2, [0])]),
+    ("c2", [(16, [0])]),
+    ("c4", [(16, [37, 74, 111, 0])]),
+]
 
 
 def other_rooflines(cfg, shapes, f, acc, n_prof, peaks):
     """The two other kernel classes of a step against their own roofs (start-to-start times, so launch gaps count):
-    attention against the sustained bf16 tensor peak (its exponentials, not the tensor pipe, pace it), and the norm
-    kernels against the measured HBM copy rate with 6 algorithmic bytes per element (fp32 in, bf16 out)."""
+    attention against the bf16 tensor peaks (its exponentials, not the tensor pipe, pace it), and the norm kernels
+    against the measured HBM copy rate with 6 algorithmic bytes per element (fp32 in, bf16 out)."""
     out = []
     if 5 in acc and acc[5][0] > 0:
         t = acc[5][0] / n_prof * 1e-3
         tf = f["attention"] / t / 1e12
-        out.append({"kernel": "attn_tc_kernel", "bound": "tensor", "achieved": tf, "peak": peaks["sustained"], "unit": "TFLOP/s",
-                    "frac": tf / peaks["sustained"], "launches_per_step": acc[5][1] // n_prof})
+        out.append({"kernel": "attn_tc_kernel", "bound": "tensor", "achieved": tf, "peak": peaks["burst"], "unit": "TFLOP/s",
+                    "frac": tf / peaks["burst"], "frac_burst": tf / peaks["burst"], "frac_sustained": tf / peaks["sustained"],
+                    "launches_per_step": acc[5][1] // n_prof})
     if 3 in acc and acc[3][0] > 0:
         t = acc[3][0] / n_prof * 1e-3
         n_norm = acc[3][1] // n_prof
@@ -144,12 +63,73 @@ def other_rooflines(cfg, shapes, f, acc, n_prof, peaks):
     return out
 
 
-def workload(cfg_name, mb, seed_shift=0):
-    cfg = S.get_config(cfg_name)
-    ci = S.configs.CONFIG_INDEX[cfg_name]
-    lg = int(np.log2(max(mb, 1)))
-    shapes = S.draw_item_shapes(cfg, mb, 3000 + 100 * ci + lg + seed_shift)
-    return cfg, shapes, 2000 + 100 * ci + lg + seed_shift
+def gemm_algorithmic_bytes(cfg, shapes):
+    """Algorithmic HBM bytes of all GEMM launches of one forward pass: every operand read once, every output written
+    once (bf16 activations and weights; the fp32 residual stream is read and written by proj and fc2; the embedding
+    reads the patch operand and writes fp32)."""
+    d, I, L = cfg["d_model"], cfg["d_mlp"], cfg["n_layers"]
+    f = flops_of(cfg, shapes)
+    T = f["tokens"]
+    up_n = (2 if cfg["mlp"] == 1 else 1) * I
+    per_layer = (2 * T * d + 2 * 3 * d * d + 2 * T * 3 * d) + (2 * T * d + 2 * d * d + 8 * T * d) \
+        + (2 * T * d + 2 * up_n * d + 2 * T * I) + (2 * T * I + 2 * d * I + 8 * T * d)
+    total = L * per_layer
+    if cfg["family"] == 2:
+        total += sum(2 * s[0] * cfg["in_channels"] + 2 * s[0] * d + 2 * s[0] * d + 4 * ((s[0] + 1) // 2) * d for s in shapes)
+        total += 2 * 3 * cfg["in_channels"] * d + 2 * 3 * d * d
+    else:
+        k = S.configs.embed_k(cfg)
+        total += (T * k * 2) + 2 * k * d + 4 * T * d
+    if cfg["head"]:
+        kin = 4 * d if cfg["head"] == 2 else d
+        r, hh, do = f["out_rows"], cfg["d_head_hidden"], cfg["d_out"]
+        total += 2 * r * kin + 2 * kin * hh + 2 * r * hh + 2 * r * hh + 2 * hh * do + 2 * r * do
+    return total
+
+
+def profile_traffic(config, micro_batch):
+    """DRAM bytes per GEMM launch (read + write, averaged over the GEMM launches of one forward pass) from the ncu
+    launch list of this workload, if a summary of it is committed under profiles/: the summary carries a line
+    `gemm_dram_bytes_per_launch = <bytes>`.  None when there is no capture of this workload."""
+    path = os.path.join(ROOT, "profiles", f"launches_{config}_mb{micro_batch}.md")
+    try:
+        with open(path) as fh:
+            for ln in fh:
+                if ln.strip().startswith("gemm_dram_bytes_per_launch"):
+                    return float(ln.split("=")[1].split()[0]), os.path.relpath(path, ROOT)
+    except (OSError, ValueError, IndexError):
+        pass
+    return None, None
+
+
+def run_sweep(main_enc, main_cfg_name, sampler):
+    """The sweep of the default run: every point timed for at least 10 steps and at least 1 s of device time, each with
+    the clock record of its own timed region."""
+    import gc
+    import torch
+    import paper_2609_31551_b200 as P
+    points = []
+    for cfg_name, plan in SWEEP:
+        if cfg_name == main_cfg_name:
+            enc, w = main_enc, None
+        else:
+            cfg = S.get_config(cfg_name)
+            w = S.make_weights(cfg)
+            enc = P.Encoder(cfg, P.weights_to_device(w))
+            del w
+        for mb, budgets in plan:
+            cfg, shapes, seed = workload(cfg_name, mb)
+            pt = Point(enc, cfg, shapes, seed)
+            for b in budgets:
+                r = time_point(pt, b, sampler, min_steps=10, min_seconds=1.0)
+                points.append(dict(config=cfg_name, micro_batch=mb, sm_budget=b if b else "all", sum_s2=pt.f["sum_s2"], **r))
+            del pt
+        if enc is not main_enc:
+            enc.close()
+            del enc
+        gc.collect()
+        torch.cuda.empty_cache()
+    return points
 
 
 # ------------------------------------------------------------------ reference arm: the oracle on host cores
@@ -227,9 +207,10 @@ def run_cuda(args):
     enc.status()
 
     # ---- value: inputs resident in HBM
-    sampler = ClockSampler(local_rank)
+    sampler = ClockSampler(local_rank).start()
+    time.sleep(0.3)                    # the sampler's first line
     barrier()
-    sampler.start()
+    mark0 = sampler.mark()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record(stream)
     for _ in range(args.steps):
@@ -280,14 +261,15 @@ def run_cuda(args):
     t1.record(s_out)
     barrier()
     ms_e2e = t0.elapsed_time(t1)
-    clocks = sampler.stop()
+    clocks = sampler.summary(mark0, sampler.mark())      # the two timed regions (resident and end-to-end)
     h2d = data.numel() * 2
     d2h = out.numel() * 2
 
     # ---- per-kernel-class timing (separate pass over the same workload, events inside the library)
     enc.enable_timing(True)
     acc = {}
-    n_prof = min(args.steps, 5)
+    n_prof = max(5, min(args.steps, 20))
+    mark1 = sampler.mark()
     for _ in range(n_prof):
         step()
         cls, kms = enc.timing_read()
@@ -296,6 +278,7 @@ def run_cuda(args):
             a[0] += m_; a[1] += 1
     enc.enable_timing(False)
     torch.cuda.synchronize()
+    clocks_prof = sampler.summary(mark1, sampler.mark())
 
     (ms, ms_e2e), (total_tokens, launches, total_items, total_flops) = R.combine(
         [ms, ms_e2e], [float(T), float(launches), float(len(shapes)), float(f["total"])], device="cuda")
@@ -309,6 +292,8 @@ def run_cuda(args):
         gemm_launch = sum(acc[c_][1] for c_ in gemm_ids if c_ in acc) / n_prof
         gemm_fl = sum(gf[c_] for c_ in gemm_ids)
         achieved = gemm_fl / (gemm_ms * 1e-3) / 1e12 if gemm_ms > 0 else 0.0
+        traffic, traffic_src = profile_traffic(args.config, args.micro_batch) if not budget else (None, None)
+        gemm_bytes = gemm_algorithmic_bytes(cfg, shapes)
         names = {0: "prep", 1: "embed_gather", 2: "gemm_embed", 3: "norm", 4: "gemm_qkv", 5: "attention", 6: "gemm_proj",
                  7: "gemm_fc1", 8: "gemm_fc2", 9: "gemm_head"}
         breakdown = {}
@@ -337,19 +322,29 @@ def run_cuda(args):
             "gpu_launches": launches,
             "clocks": clocks,
             "roofline": {"bound": "tensor", "kernel": "gemm_kernel (all GEMM launches of a step)", "achieved": achieved,
-                         "peak": peaks["sustained"], "unit": "TFLOP/s", "frac": achieved / peaks["sustained"],
-                         "peak_kind": f"sustained bf16, {peaks['source']}",
-                         # DRAM bytes of one fc1 launch of this workload from an ncu capture (profiles/gemm_fc1_c1_mb32.md):
-                         # 46.4 MB read + 97.8 MB written against 197.5 MB algorithmic (part of the output still in L2)
-                         "traffic": 143.6e6 if (args.config == "c1" and args.micro_batch == 32) else None,
-                         "traffic_note": "dram read+write bytes of one fc1 GEMM launch (ncu); algorithmic 197.5e6",
-                         "launches_per_step": gemm_launch, "avg_launch_ms": gemm_ms / max(gemm_launch, 1)},
+                         "peak": peaks["burst"], "unit": "TFLOP/s", "frac": achieved / peaks["burst"],
+                         "peak_kind": f"burst bf16, {peaks['source']}",
+                         "frac_burst": achieved / peaks["burst"], "frac_sustained": achieved / peaks["sustained"],
+                         "peak_sustained": peaks["sustained"],
+                         "traffic": traffic, "traffic_source": traffic_src,
+                         "algorithmic_bytes_per_launch": gemm_bytes / max(gemm_launch, 1),
+                         "launches_per_step": gemm_launch, "avg_launch_ms": gemm_ms / max(gemm_launch, 1),
+                         "timed_steps": n_prof, "clocks": clocks_prof},
             "roofline_other": other_rooflines(cfg, shapes, f, acc, n_prof, peaks),
             "kernel_breakdown": breakdown,
         }
+        default_point = args.config == "c1" and args.micro_batch == 32 and not budget and not args.graph and not args.split_k
+        if world == 1 and default_point and not args.no_sweep:
+            line["sweep"] = run_sweep(enc, args.config, sampler)
+            line["sweep_note"] = ("each point: 3 warm-up steps, then >= 10 steps and >= 1 s of device time between CUDA "
+                                  "events, inputs resident, with the clock record of its own timed region; fractions are "
+                                  "of the measured burst / sustained bf16 peaks")
         if world == 1 and not args.no_cpu_baseline:
             line["cpu_baseline"] = cpu_baseline(cfg, w, shapes, seed)
+        sampler.stop()
         print(json.dumps(line))
+    else:
+        sampler.stop()
     R.finish()
 
 
@@ -382,6 +377,8 @@ def main():
     ap.add_argument("--micro-batch", type=int, default=32)
     ap.add_argument("--sm-budget", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-sweep", action="store_true",
+                    help="skip the micro-batch x sm_budget sweep that the default run (c1, micro-batch 32, 1 GPU) appends")
     ap.add_argument("--split-k", action="store_true",
                     help="split the K loop of the residual GEMMs when a micro-batch has fewer tiles than SMs (latency path)")
     ap.add_argument("--graph", action="store_true",

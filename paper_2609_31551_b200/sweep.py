@@ -2,45 +2,27 @@
 
     python -m paper_2609_31551_b200.sweep --config c1 --micro-batches 1,2,4,8,16,32,64 --budgets 37,74,111,148
 
-One JSON line per point: tokens/s, items/s, TFLOP/s and the fraction of the measured bf16 peaks; inputs are the
-seeded synthetic workloads of eas_synth, resident in HBM; W warm-up steps, K timed steps between CUDA events."""
+One JSON line per point.  Every point is measured `--repeats` times (default 3), each repeat being at least
+`--min-steps` steps and `--min-seconds` of device time between CUDA events after 3 warm-up steps, with inputs (the
+seeded synthetic workloads of eas_synth) resident in HBM and the SM clock / throttle reasons sampled during the
+repeat.  The line gives the median repeat, the range over repeats, tokens/s, items/s, TFLOP/s and the fractions of the
+measured bf16 peaks; a repeat whose clock record shows a thermal or hardware slowdown is flagged."""
 from __future__ import annotations
 import argparse
 import json
 import os
+import statistics
 import sys
-
-import numpy as np
-import torch
 
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
-import bench  # noqa: E402  (FLOP model, workload recipe, measured peaks)
 import eas_synth as S  # noqa: E402
 from . import binding as B  # noqa: E402
+from . import measure as M  # noqa: E402
 
-
-def run_point(enc, cfg, shapes, seed, budget, steps, warmup):
-    items = S.make_items(cfg, shapes, seed)
-    data, offsets = B.pack_items(items)
-    cu = np.concatenate([[0], np.cumsum([S.tokens_per_item(cfg, s) for s in shapes])]).astype(np.int32)
-    cu_dev = torch.from_numpy(cu).cuda()
-    f = bench.flops_of(cfg, shapes)
-    out = torch.empty((f["out_rows"], cfg["d_out"]), dtype=torch.bfloat16, device="cuda")
-    for _ in range(warmup):
-        enc.encode_microbatch(data, shapes, offsets, cu, cu_seqlens_dev=cu_dev, sm_budget=budget, out=out)
-    enc.status()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    for _ in range(steps):
-        enc.encode_microbatch(data, shapes, offsets, cu, cu_seqlens_dev=cu_dev, sm_budget=budget, out=out)
-    e1.record()
-    torch.cuda.synchronize()
-    enc.status()
-    ms = e0.elapsed_time(e1) / steps
-    return ms, f
+BAD_REASONS = {"hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown"}
 
 
 def main():
@@ -48,30 +30,39 @@ def main():
     ap.add_argument("--config", default="c1")
     ap.add_argument("--micro-batches", default="1,2,4,8,16,32,64")
     ap.add_argument("--budgets", default="37,74,111,148")
-    ap.add_argument("--steps", type=int, default=5)
-    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--repeats", type=int, default=3)
+    ap.add_argument("--min-steps", type=int, default=10)
+    ap.add_argument("--min-seconds", type=float, default=0.5)
     ap.add_argument("--max-tokens", type=int, default=400000, help="skip points with more encoder tokens than this")
     a = ap.parse_args()
-    peaks = bench.measured_peaks()
+    import torch
+    peaks = M.measured_peaks()
     cfg = S.get_config(a.config)
     w = S.make_weights(cfg)
     enc = B.Encoder(cfg, B.weights_to_device(w))
     del w
+    sampler = M.ClockSampler(torch.cuda.current_device()).start()
     for mb in [int(x) for x in a.micro_batches.split(",")]:
-        _, shapes, seed = bench.workload(a.config, mb)
+        _, shapes, seed = M.workload(a.config, mb)
         T = sum(S.tokens_per_item(cfg, s) for s in shapes)
         if T > a.max_tokens:
             print(json.dumps({"config": a.config, "micro_batch": mb, "skipped": f"{T} tokens > --max-tokens"}))
             continue
+        pt = M.Point(enc, cfg, shapes, seed)
         for budget in [int(x) for x in a.budgets.split(",")]:
-            ms, f = run_point(enc, cfg, shapes, seed, budget, a.steps, a.warmup)
-            tf = f["total"] / ms / 1e9
-            print(json.dumps({"config": a.config, "micro_batch": mb, "sm_budget": budget, "tokens": f["tokens"],
-                              "sum_s2": f["sum_s2"], "ms_per_step": round(ms, 4),
-                              "tokens_per_s": round(f["tokens"] / ms * 1e3, 1), "items_per_s": round(mb / ms * 1e3, 2),
-                              "tflops": round(tf, 1), "attn_flop_share": round(f["attention"] / f["total"], 3),
-                              "frac_burst": round(tf / peaks["burst"], 4), "frac_sustained": round(tf / peaks["sustained"], 4),
-                              "peaks": peaks["source"]}), flush=True)
+            runs = [M.time_point(pt, budget, sampler, min_steps=a.min_steps, min_seconds=a.min_seconds) for _ in range(a.repeats)]
+            runs.sort(key=lambda r: r["ms_per_step"])
+            med = runs[len(runs) // 2]
+            reasons = sorted(set(x for r in runs for x in r["clocks"]["reasons"]))
+            mhz = [r["clocks"]["sm_mhz"] for r in runs if r["clocks"].get("sm_mhz")]
+            line = dict(config=a.config, micro_batch=mb, sm_budget=budget, sum_s2=pt.f["sum_s2"], **med)
+            line.update(repeats=len(runs), ms_min=runs[0]["ms_per_step"], ms_max=runs[-1]["ms_per_step"],
+                        sm_mhz_median=statistics.median(mhz) if mhz else None, reasons=reasons,
+                        rejected=bool(BAD_REASONS & set(reasons)), peaks=peaks["source"])
+            line.pop("clocks", None)
+            print(json.dumps(line), flush=True)
+        del pt
+    sampler.stop()
 
 
 if __name__ == "__main__":

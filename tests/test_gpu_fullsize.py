@@ -52,6 +52,14 @@ def test_c1_full_depth_two_images(profile, seed):
     rel, mabs = G.assert_parity(got, ref, f"c1 {profile}")
     G.record_margin("c1 mb2 full depth", profile, seed, rel, mabs)
     print(f"c1 {profile} full depth seed {seed}:", rel, mabs)
+    # the same pass with fp32 output (EAS_OUT_FP32): what remains of the error without the output rounding
+    import paper_2609_31551_b200 as P
+    enc32 = P.Encoder(dict(cfg, out_dtype=1), enc._weights)
+    got32, dev32 = G.run_gpu(enc32, cfg, items)
+    assert dev32.dtype == torch.float32
+    rel32, mabs32 = G.assert_parity(got32, ref, f"c1 {profile} fp32 out")
+    G.record_margin("c1 mb2 full depth, fp32 output", profile, seed, rel32, mabs32)
+    assert mabs32 <= mabs
 
 
 @pytest.mark.parametrize("profile,seed", [("plain", 2203), ("sharp", 2203), ("plain", 2213)])

@@ -85,23 +85,27 @@ def test_gemm_tile_shapes_agree_bit_for_bit_with_large_distinct_biases(act, out_
     A, W = _dev(_bf16_exact(rng, (M, K))), _dev(_bf16_exact(rng, (N, K), 0.02))
     bias = np.repeat(np.arange(N // 256, dtype=np.float32) * 8.0 - 24.0, 256) + rng.standard_normal(N).astype(np.float32)
     b = _dev(S.round_to_bf16(bias))
-    resid = torch.from_numpy(rng.standard_normal((M, N)).astype(np.float32)).cuda() if out_fp32 else None
-    ref, st = P.kernel_gemm(A, W, b, act=act, out_fp32=out_fp32, resid=resid, sm_budget=2, tile_shape=1)
-    torch.cuda.synchronize()
-    assert int(st[0]) == 0
+    x0 = torch.from_numpy(rng.standard_normal((M, N)).astype(np.float32)).cuda() if out_fp32 else None
+
+    def run(budget, shape):
+        # the fp32 case is the residual update in place (x += A W^T + b), the only fp32 form the wide tile serves
+        x = x0.clone() if out_fp32 else None
+        out, st = P.kernel_gemm(A, W, b, act=act, out_fp32=out_fp32, resid=x, out=x, sm_budget=budget, tile_shape=shape)
+        torch.cuda.synchronize()
+        assert int(st[0]) == 0
+        return out
+
+    ref = run(2, 1)
     y = O.linear(O._t(A.float().cpu().numpy()), O._t(W.float().cpu().numpy()), O._t(b.float().cpu().numpy()))
     if act == 1:
         y = O.gelu(y)
     if out_fp32:
-        y = y + resid.double().cpu()
+        y = y + x0.double().cpu()
     assert (ref.double().cpu() - y).abs().max() <= 2.0 ** -7 * float(y.abs().max())
     for shape in (2, 3):
         for budget in (2, 6, 148):
             for _ in range(3):
-                out, st = P.kernel_gemm(A, W, b, act=act, out_fp32=out_fp32, resid=resid, sm_budget=budget, tile_shape=shape)
-                torch.cuda.synchronize()
-                assert int(st[0]) == 0
-                assert torch.equal(out, ref), (shape, budget)
+                assert torch.equal(run(budget, shape), ref), (shape, budget)
 
 
 def test_gemm_wide_tile_is_refused_where_it_does_not_exist():
