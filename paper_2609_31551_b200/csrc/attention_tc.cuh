@@ -183,6 +183,9 @@ __device__ __forceinline__ void tmem_ld_32x32_at(uint32_t taddr, uint32_t (&r)[N
 // 2^x for a pair of arguments on the FMA pipe instead of the special-function unit: x = n + f with n = rint(x)
 // (magic-number rounding), 2^f by a cubic fitted on [-0.5, 0.5] (relative error below 8e-5, far under the bf16
 // rounding of P), then n is added to the exponent field.  Arguments are clamped at -126 (result ~1e-38 instead of 0).
+#ifndef EAS_ATTN_MAX_CHAINS
+#define EAS_ATTN_MAX_CHAINS 4      // independent chains of the row-maximum reduction (a power of two)
+#endif
 #ifndef EAS_ATTN_POLY_OF_4
 #define EAS_ATTN_POLY_OF_4 1      // of every 4 pairs of probabilities, this many take the polynomial path
 #endif
@@ -708,13 +711,19 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_tc_kernel(const __grid_con
 #pragma unroll
           for (int i = 0; i < KEYS; ++i) if (i >= valid) sr[i] = 0xff800000u;   // -inf
         }
-        float mx0 = -INFINITY, mx1 = -INFINITY;
+        // row maximum: EAS_ATTN_MAX_CHAINS independent chains of 3-input maxima (a chain is a string of dependent
+        // instructions: more, shorter chains hide their latency behind each other), folded at the end
+        float mxc[EAS_ATTN_MAX_CHAINS];
 #pragma unroll
-        for (int i = 0; i < KEYS; i += 4) {
-          mx0 = fmax3(mx0, __uint_as_float(sr[i]), __uint_as_float(sr[i + 1]));
-          mx1 = fmax3(mx1, __uint_as_float(sr[i + 2]), __uint_as_float(sr[i + 3]));
-        }
-        const float mx = fmaxf(mx0, mx1);
+        for (int c = 0; c < EAS_ATTN_MAX_CHAINS; ++c) mxc[c] = -INFINITY;
+#pragma unroll
+        for (int i = 0; i < KEYS; i += 2)
+          mxc[(i / 2) % EAS_ATTN_MAX_CHAINS] = fmax3(mxc[(i / 2) % EAS_ATTN_MAX_CHAINS], __uint_as_float(sr[i]), __uint_as_float(sr[i + 1]));
+#pragma unroll
+        for (int w2 = EAS_ATTN_MAX_CHAINS / 2; w2 >= 1; w2 >>= 1)
+#pragma unroll
+          for (int c = 0; c < w2; ++c) mxc[c] = fmaxf(mxc[c], mxc[c + w2]);
+        const float mx = mxc[0];
         ATTN_STAMP(3);
         // reference maximum: moves only when the row maximum grew by more than the threshold
         float corr = 1.0f;

@@ -20,6 +20,7 @@
 #include "attention_mma.cuh"
 #include "attention_tc.cuh"
 #include "elementwise.cuh"
+#include "embed_gemm.cuh"
 #include "gemm.cuh"
 
 using namespace eas;
@@ -148,6 +149,7 @@ struct eas_encoder {
   int sm_count = 0;
   int hd = 0;
   int embed_k = 0, embed_k_pad = 0;
+  const uint32_t* embed_table = nullptr;   // where each pixel pair of a patch vector comes from (embed_gemm.cuh)
   Linear embed, conv1, conv2, head1, head2;
   const bf16 *cls = nullptr, *pos = nullptr, *eng = nullptr, *enb = nullptr, *fng = nullptr, *fnb = nullptr, *hng = nullptr;
   std::vector<Layer> layers;
@@ -222,7 +224,8 @@ extern "C" size_t eas_encoder_weight_arena_bytes(const eas_arch_config* c) {
   if (check_cfg(c) != EAS_OK) return 0;
   size_t total = 1024;
   const size_t d = c->d_model, I = c->d_mlp;
-  if (c->family != EAS_FAMILY_AUDIO_CONV) total += align_up(d * align_up(embed_k_of(c), 64) * 2, 1024);
+  if (c->family != EAS_FAMILY_AUDIO_CONV)   // padded patch matrix + the embedding kernel's pair table
+    total += align_up(d * align_up(embed_k_of(c), 64) * 2, 1024) + align_up(align_up(embed_k_of(c), 64) * 2, 1024);
   if (c->pos == EAS_POS_ROPE_2D) total += c->n_layers * (align_up(3 * d * d * 2, 1024) + align_up(3 * d * 2, 1024));
   if (c->mlp == EAS_MLP_SWIGLU) total += c->n_layers * (align_up(2 * I * d * 2, 1024) + align_up(2 * I * 2, 1024));
   return total;
@@ -422,6 +425,8 @@ extern "C" eas_status eas_encoder_create(const eas_arch_config* arch, const eas_
   } else {
     e->embed_k = embed_k_of(&c);
     e->embed_k_pad = static_cast<int>(align_up(e->embed_k, 64));
+    if (e->embed_k_pad > 4096 || c.patch > 255 || c.temporal_patch > 255 || c.in_channels > 255)
+      return fail(EAS_ERR_UNSUPPORTED, "patch vector of %d elements (at most %d; patch, temporal patch and channels at most 255)", e->embed_k, 4096);
     const bf16* w = nullptr;
     EAS_TRY(wi.get("embed.w", {d, e->embed_k}, &w));
     EAS_TRY(wi.get("embed.b", {d}, &e->embed.b));
@@ -430,6 +435,11 @@ extern "C" eas_status eas_encoder_create(const eas_arch_config* arch, const eas_
     EAS_TRY(relayout(dst, w, nullptr, d, e->embed_k, e->embed_k_pad, 0, 0, 0));
     e->embed.w = dst; e->embed.N = d; e->embed.K = e->embed_k_pad;
     EAS_TRY(finish_linear(e->embed));
+    uint32_t* table = static_cast<uint32_t*>(arena.take(static_cast<size_t>(e->embed_k_pad) * 2));
+    if (table == nullptr) return fail(EAS_ERR_WORKSPACE, "weight arena exhausted");
+    embed_table_kernel<<<4, 256>>>(table, e->embed_k, e->embed_k_pad, c.patch, c.temporal_patch);
+    CUDA_TRY(cudaGetLastError());
+    e->embed_table = table;
   }
   if (c.has_cls) EAS_TRY(wi.get("cls", {d}, &e->cls));
   if (c.pos == EAS_POS_TABLE) EAS_TRY(wi.get("pos", {c.max_pos, d}, &e->pos));
@@ -526,7 +536,7 @@ extern "C" int32_t eas_encoder_last_launch_count(const eas_encoder* enc) { retur
 // ------------------------------------------------------------------------------------ workspace plan
 namespace {
 struct Plan {
-  size_t status, x, n, qkv, o, a, embed_a, row_map, pos_idx, head_src, rope, mel_pad, h1_pad, conv1_map, part, total;
+  size_t status, x, n, qkv, o, a, row_map, pos_idx, head_src, rope, mel_pad, h1_pad, conv1_map, part, total;
   int splits_proj, splits_fc2;     // split-K factors of the two residual GEMMs of a block (1: off)
   int64_t part_rows;               // rows of one split's region of the partial-sum scratch
   int64_t T, embed_rows, padded_rows, out_rows;
@@ -562,7 +572,6 @@ static Plan make_plan(const eas_encoder* e, int64_t T, int n_items) {
   p.o = take(T * d * 2);
   const size_t a_elems = std::max<size_t>(T * static_cast<size_t>(c.d_mlp), static_cast<size_t>(p.out_rows) * std::max(c.d_head_hidden, 0));
   p.a = take(a_elems * 2);
-  p.embed_a = take(audio ? 0 : static_cast<size_t>(p.embed_rows) * e->embed_k_pad * 2);
   p.row_map = take(static_cast<size_t>(p.embed_rows) * 4);
   p.pos_idx = take(static_cast<size_t>(p.embed_rows) * 4);
   p.head_src = take(static_cast<size_t>(T) * 4);
@@ -947,6 +956,8 @@ static eas_status encode_impl(eas_encoder* e, const eas_packed_inputs* in, void*
       if (h % unit != 0 || w % unit != 0) return fail(EAS_ERR_INVALID_ARG, "item %d: height/width must be multiples of %d", i, unit);
       if (f % c.temporal_patch != 0) return fail(EAS_ERR_INVALID_ARG, "item %d: frames must be a multiple of %d", i, c.temporal_patch);
       if (c.temporal_patch == 1 && f != 1) return fail(EAS_ERR_INVALID_ARG, "item %d: an image encoder takes one frame", i);
+      if (static_cast<long long>(f) * c.in_channels * h * w >= (1LL << 31))
+        return fail(EAS_ERR_UNSUPPORTED, "item %d has 2^31 or more elements", i);
       const int patches = (f / c.temporal_patch) * (h / c.patch) * (w / c.patch);
       expect = patches + (c.has_cls ? 1 : 0);
       aux += patches;
@@ -968,7 +979,6 @@ static eas_status encode_impl(eas_encoder* e, const eas_packed_inputs* in, void*
   bf16* qkv = reinterpret_cast<bf16*>(ws + pl.qkv);
   bf16* obuf = reinterpret_cast<bf16*>(ws + pl.o);
   bf16* abuf = reinterpret_cast<bf16*>(ws + pl.a);
-  bf16* embed_a = reinterpret_cast<bf16*>(ws + pl.embed_a);
   int* row_map = reinterpret_cast<int*>(ws + pl.row_map);
   int* pos_idx = reinterpret_cast<int*>(ws + pl.pos_idx);
   int* head_src = reinterpret_cast<int*>(ws + pl.head_src);
@@ -1029,26 +1039,30 @@ static eas_status encode_impl(eas_encoder* e, const eas_packed_inputs* in, void*
     EAS_TRY(mark(e, EAS_KC_GEMM_EMBED, stream));
     EAS_TRY(launch_gemm(g2, budget, stream, status)); ++launches;
   } else {
-    Im2colParams ip{};
-    ip.data = static_cast<const bf16*>(in->data); ip.a = embed_a;
-    ip.n_patches = static_cast<int>(pl.embed_rows); ip.k = e->embed_k; ip.k_pad = e->embed_k_pad;
-    ip.channels = c.in_channels; ip.patch = c.patch; ip.tpatch = c.temporal_patch;
-    ip.merge_order = c.family == EAS_FAMILY_VIT_ROPE_MERGER ? 1 : 0;
-    ip.items = items;
+    // patch embedding: the im2col gather is the GEMM's A producer (no patch matrix in global memory)
+    EmbedGemmParams gp{};
+    gp.tma_w = e->embed.tmap;
+    gp.data = static_cast<const bf16*>(in->data); gp.bias = e->embed.b; gp.x = x;
+    gp.row_map = row_map;
+    if (c.pos == EAS_POS_TABLE) { gp.pos_idx = pos_idx; gp.pos = e->pos; }
+    gp.n_patches = static_cast<int>(pl.embed_rows); gp.N = d; gp.k = e->embed_k; gp.k_pad = e->embed_k_pad;
+    gp.channels = c.in_channels; gp.patch = c.patch; gp.tpatch = c.temporal_patch;
+    gp.merge_order = c.family == EAS_FAMILY_VIT_ROPE_MERGER ? 1 : 0;
+    gp.pairs_ok = (c.patch % 2 == 0 && (reinterpret_cast<uintptr_t>(in->data) & 3) == 0) ? 1 : 0;
+    for (int i = 0; i < n && gp.pairs_ok; ++i)
+      if ((in->item_offset[i] & 1) != 0 || (in->item_shape[3 * i + 2] & 1) != 0) gp.pairs_ok = 0;
+    gp.table = e->embed_table;
+    gp.status = status;
+    gp.items = items;
     static OncePerDevice once;
     if (once.first()) {
-      CUDA_TRY(cudaFuncSetAttribute(im2col_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kOnePerSmSmem));
+      CUDA_TRY(cudaFuncSetAttribute(embed_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kEgSmemBytes));
       once.settled();
     }
-    EAS_TRY(mark(e, EAS_KC_EMBED_GATHER, stream));
-    EAS_TRY(launch_kernel(im2col_kernel, budget, 512, kOnePerSmSmem, stream, ip));
-    ++launches;
-    GemmCall g;
-    g.A = embed_a; g.a_run = e->embed_k_pad; g.a_row_elems = e->embed_k_pad; g.a_rows = pl.embed_rows; g.M = static_cast<int>(pl.embed_rows);
-    g.lin = &e->embed; g.out_fp32 = 1; g.out = x; g.ldo = d; g.row_map = row_map;
-    if (c.pos == EAS_POS_TABLE) { g.pos_idx = pos_idx; g.pos = e->pos; }
+    const int tiles = static_cast<int>((pl.embed_rows + 127) / 128);     // a CTA owns whole blocks of 128 patches
     EAS_TRY(mark(e, EAS_KC_GEMM_EMBED, stream));
-    EAS_TRY(launch_gemm(g, budget, stream, status)); ++launches;
+    EAS_TRY(launch_kernel(embed_gemm_kernel, std::min(budget, tiles), kEgThreads, kEgSmemBytes, stream, gp));
+    ++launches;
   }
   if (c.embed_norm) {
     NormParams np{x, x, e->eng, e->enb, nullptr, static_cast<int>(T), d, c.norm_eps};

@@ -1,6 +1,6 @@
 // HBM-bound kernels of the encoder: row normalisation (LayerNorm / RMSNorm / plain cast) with an
-// optional row gather, patch gathering (im2col), per-call tables (row maps, rotary table), audio
-// staging, and the one-off weight re-layouts done at create time.
+// optional row gather, per-call tables (row maps, rotary table), audio staging, and the one-off weight
+// re-layouts done at create time.  (Patch gathering is part of the embedding GEMM: embed_gemm.cuh.)
 // All per-call kernels are persistent grid-stride loops launched with `sm_budget` CTAs.
 #pragma once
 #include "ptx.cuh"
@@ -131,67 +131,6 @@ __global__ void __launch_bounds__(512, 1) norm_kernel(const NormParams p) {
         reinterpret_cast<uint2*>(reinterpret_cast<bf16*>(p.y) + static_cast<long long>(row) * p.d)[i * 32 + lane] = o2;
       }
     }
-  }
-}
-
-// ------------------------------------------------------------------------------- patch gather
-struct Im2colParams {
-  const bf16* data;      // packed items
-  bf16* a;               // [n_patches, k_pad]
-  int n_patches, k, k_pad;
-  int channels, patch, tpatch;
-  int merge_order;       // 0: raster order; 1: merge-group-major order (2x2 groups consecutive)
-  ItemTable items;       // aux_start = patch-row prefix
-};
-
-// One thread copies one run of P horizontally adjacent pixels (one row of one channel of one patch) or one
-// run of the zero padding behind the patch; the item lookup and the index arithmetic are paid once per run.
-__global__ void __launch_bounds__(512, 1) im2col_kernel(const __grid_constant__ Im2colParams p) {
-  const int P = p.patch;
-  const int runs = p.channels * p.tpatch * P;                  // pixel runs per patch
-  const int pad_runs = (p.k_pad - p.k + P - 1) / P;            // zero runs per patch
-  const int per_patch = runs + pad_runs;
-  const long long total = static_cast<long long>(p.n_patches) * per_patch;
-  pdl_launch_dependents();
-  pdl_wait();
-  for (long long idx = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x; idx < total;
-       idx += static_cast<long long>(gridDim.x) * blockDim.x) {
-    const int m = static_cast<int>(idx / per_patch);
-    const int run = static_cast<int>(idx - static_cast<long long>(m) * per_patch);
-    bf16* dst = p.a + static_cast<long long>(m) * p.k_pad;
-    if (run >= runs) {
-      const int e0 = p.k + (run - runs) * P;
-      for (int e = e0; e < min(e0 + P, p.k_pad); ++e) dst[e] = __float2bfloat16(0.f);
-      continue;
-    }
-    const int it = find_item(p.items.aux_start, p.items.n_items, m);
-    const int local = m - p.items.aux_start[it];
-    const int H = p.items.height[it], W = p.items.width[it];
-    const int gh = H / P, gw = W / P;
-    const int t = local / (gh * gw);
-    const int rem = local - t * gh * gw;
-    int r, c;
-    if (p.merge_order) {
-      const int grp = rem >> 2, within = rem & 3;
-      const int hb = grp / (gw >> 1), wb = grp - hb * (gw >> 1);
-      r = 2 * hb + (within >> 1);
-      c = 2 * wb + (within & 1);
-    } else {
-      r = rem / gw;
-      c = rem - r * gw;
-    }
-    // run order inside a patch row: (channel, frame-in-patch, py), then px contiguous
-    const int py = run % P;
-    const int f = (run / P) % p.tpatch;
-    const int ch = run / (P * p.tpatch);
-    long long off = p.items.offset[it];
-    if (p.tpatch > 1 || p.items.frames[it] > 1)
-      off += ((static_cast<long long>(t * p.tpatch + f) * p.channels + ch) * H + (r * P + py)) * W + c * P;
-    else
-      off += (static_cast<long long>(ch) * H + (r * P + py)) * W + c * P;
-    const bf16* src = p.data + off;
-    bf16* d = dst + run * P;
-    for (int px = 0; px < P; ++px) d[px] = src[px];
   }
 }
 

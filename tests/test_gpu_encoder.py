@@ -128,3 +128,55 @@ def test_split_k_parity_all_families(case):
     G.assert_parity(got, ref, case + " split K")
     _, again = G.run_gpu(enc, cfg, items, sm_budget=37)
     assert torch.equal(dev, again)
+
+
+EMBED_CASES = {
+    "c0": [(1, 224, 224), (1, 32, 48)],
+    "c1": [(1, 336, 336)] * 2,
+    "c2": [(1, 56, 84), (1, 364, 140), (1, 28, 28), (1, 224, 1344)],
+    "c3": [(4, 56, 56), (2, 112, 84), (6, 28, 28)],
+}
+
+
+@pytest.mark.parametrize("name", list(EMBED_CASES))
+def test_fused_patch_embedding_alone(name):
+    """An encoder without transformer blocks is the embedding (patch gather fused into the GEMM, bias, position
+    rows, CLS) followed by the connector: the gather's index arithmetic for images, clips, raster and
+    merge-group-major patch order, several items of different sizes and a ragged last tile, against the oracle."""
+    over = dict(n_layers=0)
+    if name in ("c0", "c1"):
+        over["max_pos"] = 600
+    cfg = S.get_config(name, **over)
+    if name == "c0":
+        cfg = dict(cfg, out_dtype=1)           # final LayerNorm in fp32: nothing but the embedding's own rounding is left
+    w, enc = _make(cfg)
+    shapes = EMBED_CASES[name]
+    items = S.make_items(cfg, shapes, seed=4100)
+    ref, _, _ = O.encode_microbatch(cfg, w, items)
+    got, dev = G.run_gpu(enc, cfg, items)
+    rel, mabs = G.assert_parity(got, ref, f"{name} embedding only")
+    if name == "c0":
+        assert rel < 2e-3, rel                 # bf16 operands with fp32 accumulation: far inside the tolerance
+    for budget in (1, 5, 37):
+        _, b = G.run_gpu(enc, cfg, items, sm_budget=budget)
+        assert torch.equal(b, dev), budget
+
+
+def test_fused_patch_embedding_with_odd_item_offsets():
+    """Item offsets that are odd element counts break the 4-byte alignment of pixel pairs: the gather then loads
+    single elements.  Same values, same accumulation order: the result must be the same bytes."""
+    import paper_2609_31551_b200 as P
+    cfg = S.get_config("c2", n_layers=1)
+    w, enc = _make(cfg)
+    shapes = [(1, 56, 84), (1, 28, 140)]
+    items = S.make_items(cfg, shapes, seed=4200)
+    _, want = G.run_gpu(enc, cfg, items)
+    flat = [torch.from_numpy(np.ascontiguousarray(it).reshape(-1)).to(torch.bfloat16) for it in items]
+    offsets = [1, 1 + flat[0].numel() + 2]     # 1 and an odd number: both items start on odd elements
+    buf = torch.zeros(offsets[1] + flat[1].numel() + 8, dtype=torch.bfloat16)
+    for f, o in zip(flat, offsets):
+        buf[o:o + f.numel()] = f
+    cu = G.cu_seqlens_of(cfg, items)
+    out = enc.encode_microbatch(buf.cuda(), shapes, offsets, cu)
+    enc.status()
+    assert torch.equal(out, want)
