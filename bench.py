@@ -132,6 +132,15 @@ def run_sweep(main_enc, main_cfg_name, sampler):
     return points
 
 
+def config_of(args, n_items, tokens, world):
+    """The `config` object of a line: the same for both arms (the reference arm times the oracle on this workload)."""
+    return {"workload": f"{args.config} micro-batch {args.micro_batch}", "items_per_step": n_items,
+            "tokens_per_step": tokens, "sm_budget": args.sm_budget if args.sm_budget else "all",
+            "l2": "working set (weights + activations) larger than L2; no flush",
+            "parallelism": "replicas" if world > 1 else "single",
+            "launch": ("cuda graph replay" if args.graph else "one launch per kernel") + (", split K" if args.split_k else "")}
+
+
 # ------------------------------------------------------------------ reference arm: the oracle on host cores
 def run_reference(args):
     import torch
@@ -154,11 +163,11 @@ def run_reference(args):
     line = {"impl": "reference", "metric": "encoder_tokens_per_sec", "value": val, "unit": "tokens/s", "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": f"{args.config} micro-batch {args.micro_batch}", "items_per_step": len(shapes),
-                       "tokens_per_step": sum(S.tokens_per_item(cfg, s) for s in shapes), "sm_budget": "host cores",
-                       "sampled": "each step encodes 1 item of the micro-batch (bounded sample)"},
+            "config": config_of(args, len(shapes), sum(S.tokens_per_item(cfg, s) for s in shapes),
+                                int(os.environ.get("WORLD_SIZE", "1"))),
             "cpu_baseline": {"value": val, "unit": "tokens/s", "cores": torch.get_num_threads(), "kind": "oracle",
-                             "sample": f"1 item ({f['tokens']} tokens) of the {args.config} micro-batch per step"},
+                             "sample": f"each step encodes 1 item ({f['tokens']} tokens) of the {args.config} micro-batch "
+                                       "on the host cores (bounded sample)"},
             "e2e": {"value": val, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
     print(json.dumps(line))
 
@@ -307,11 +316,7 @@ def run_cuda(args):
             "metric": "encoder_tokens_per_sec", "value": total_tokens * args.steps / (ms * 1e-3), "unit": "tokens/s",
             "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": step_ms,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": f"{args.config} micro-batch {args.micro_batch}", "items_per_step": len(shapes),
-                       "tokens_per_step": T, "sm_budget": budget if budget else "all",
-                       "l2": "working set (weights + activations) larger than L2; no flush",
-                       "parallelism": "replicas" if world > 1 else "single",
-                       "launch": ("cuda graph replay" if args.graph else "one launch per kernel") + (", split K" if args.split_k else "")},
+            "config": config_of(args, len(shapes), T, world),
             "items_per_sec": total_items * args.steps / (ms * 1e-3),
             "tflops": total_flops / (step_ms * 1e-3) / 1e12,
             "frac_of_bf16_peak": {"burst_measured": f["total"] / (step_ms * 1e-3) / 1e12 / peaks["burst"],
