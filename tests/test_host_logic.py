@@ -135,3 +135,49 @@ def test_replica_bookkeeping_world_size_2_gloo():
         assert ms == [11.0, 5.0]            # slowest rank per measurement
         assert sums == [300.0, 14.0]        # work adds up over replicas
         assert shift == 1000 * rank         # every replica draws its own micro-batches
+
+
+def test_flop_model_against_closed_forms():
+    """The benchmark's algorithmic FLOP count against the per-item figures that follow from the layer shapes:
+    c1 704 MFLOP per token (406 GFLOP per 336x336 image), c4 2.27 TFLOP per 3000-frame clip; attention is 4 d S^2 per
+    item and layer; nothing is counted for padding."""
+    from paper_2609_31551_b200 import measure as M
+    c1 = S.get_config("c1")
+    f = M.flops_of(c1, [(1, 336, 336)])
+    assert f["tokens"] == 577 and f["out_rows"] == 576
+    assert abs(f["total"] / 1e9 - 406) < 2
+    lin = 24 * 577 * (8 * 1024 * 1024 + 4 * 1024 * 4096)
+    assert f["attention"] == 24 * 4 * 1024 * 577 * 577
+    assert f["linear"] == lin + 2 * 576 * 588 * 1024 + 2 * 576 * (1024 * 4096 + 4096 * 4096)
+    two = M.flops_of(c1, [(1, 336, 336)] * 2)
+    assert two["total"] == 2 * f["total"]                       # items never interact
+    c4 = S.get_config("c4")
+    f4 = M.flops_of(c4, [(3000, 128, 1)])
+    assert f4["tokens"] == 1500 and abs(f4["total"] / 1e12 - 2.27) < 0.02
+    assert M.flops_of(c4, [(2999, 128, 1)])["tokens"] == 1500    # odd frame counts: ceil(n / 2) tokens
+    c3 = S.get_config("c3")
+    f3 = M.flops_of(c3, [(16, 448, 448)])
+    assert f3["tokens"] == 8192 and abs(f3["total"] / 1e12 - 24.9) < 0.2
+    by = M.gemm_flops_by_class(c1, [(1, 336, 336)])
+    assert sum(by.values()) == f["total"]
+
+
+def test_reference_arm_prints_the_contract_line():
+    """`bench.py --impl reference` (the oracle on host cores) prints one JSON line with the keys the benchmark contract
+    names and the same `config` object the CUDA arm prints for the same arguments."""
+    import json
+    import subprocess
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--config", "c0",
+                          "--micro-batch", "4", "--steps", "1", "--warmup", "0"], capture_output=True, text=True, timeout=600)
+    assert out.returncode == 0, out.stderr[-2000:]
+    line = json.loads(out.stdout.strip().splitlines()[-1])
+    for key in ("impl", "metric", "value", "unit", "n_gpus", "steps", "warmup", "ms_per_step", "higher_is_better", "scaling",
+                "vs_baseline", "dtype", "data", "config", "cpu_baseline", "e2e"):
+        assert key in line, key
+    assert line["impl"] == "reference" and line["dtype"] == "f64" and line["vs_baseline"] is None
+    assert line["cpu_baseline"]["kind"] == "oracle" and line["cpu_baseline"]["cores"] >= 1
+    assert line["e2e"]["h2d_bytes_per_step"] == 0 and line["e2e"]["d2h_bytes_per_step"] == 0
+    import argparse
+    import bench
+    args = argparse.Namespace(config="c0", micro_batch=4, sm_budget=0, graph=False, split_k=False)
+    assert line["config"] == bench.config_of(args, 4, 784, 1)
