@@ -226,13 +226,15 @@ def test_attention_head_dim_80_key_tile_edges(H):
 
 
 @pytest.mark.parametrize("hd", [64, 80])
-@pytest.mark.parametrize("case", ["rising", "falling", "peaked", "uniform", "tiny_scores"])
+@pytest.mark.parametrize("case", ["rising", "falling", "steep_rising", "late_spike", "peaked", "uniform", "tiny_scores"])
 def test_attention_softmax_degenerate_score_patterns(hd, case):
     """The online softmax across key tiles under score patterns that stress it: scores that rise with the key index
     (the running maximum grows in every tile, every earlier partial sum is rescaled), scores that fall (the first
     tile holds the maximum, later tiles underflow), one dominant key per query with score gaps of hundreds (the
     output is that key's value row), equal keys (the output is the mean of the values: a closed form), and scores
-    of magnitude 1e-3."""
+    of magnitude 1e-3.  Two more put a score far above everything seen so far into a LATER key tile, hundreds of
+    octaves above the running maximum, where 2^(score - stale maximum) overflows fp32: a ramp that climbs thousands
+    per tile, and one spike key per item among small scores."""
     import paper_2609_31551_b200 as P
     H, lens = 2, [700, 130]
     T, d = sum(lens), H * hd
@@ -246,6 +248,14 @@ def test_attention_softmax_degenerate_score_patterns(hd, case):
         # 0 ... 87 (hd 64) or 98 (hd 80) over 700 keys
         q[:] = 1.0
         k[:] = (pos / 64.0) * (1.0 if case == "rising" else -1.0)
+    elif case == "steep_rising":
+        q[:] = 1.0
+        k[:] = pos * 4.0
+    elif case == "late_spike":
+        q[:] = 1.0
+        k *= 0.125
+        k[500] = 50.0                       # item 0, fourth key tile
+        k[700 + 129] = 50.0                 # item 1, second key tile (its last key)
     elif case == "peaked":
         q *= 6.0
         k *= 6.0
