@@ -196,6 +196,8 @@ def run_cuda(args):
     budget = args.sm_budget
     if args.split_k:
         enc.set_split_k(True)          # before any workspace is sized
+    if args.norm_fold:
+        enc.set_norm_fold(True)
     if args.graph:
         # the launch-overhead path: captured forward passes need a stream of their own
         torch.cuda.set_stream(torch.cuda.Stream())
@@ -386,6 +388,8 @@ def main():
                     help="skip the micro-batch x sm_budget sweep that the default run (c1, micro-batch 32, 1 GPU) appends")
     ap.add_argument("--split-k", action="store_true",
                     help="split the K loop of the residual GEMMs when a micro-batch has fewer tiles than SMs (latency path)")
+    ap.add_argument("--norm-fold", action="store_true",
+                    help="fold the blocks' normalisations into the GEMMs around them instead of one kernel per norm1 / norm2")
     ap.add_argument("--graph", action="store_true",
                     help="replay captured forward passes (CUDA graphs): the launch-overhead path for small micro-batches")
     args = ap.parse_args()

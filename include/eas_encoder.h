@@ -190,6 +190,17 @@ eas_status eas_encoder_set_attention_impl(eas_encoder* enc, int32_t impl);
  * partial sums need scratch): set it before sizing the workspace. */
 eas_status eas_encoder_set_split_k(eas_encoder* enc, int32_t on);
 
+/* Folded normalisation (default on).  A block's norm1 / norm2 (Section 2.1: pre-norm transformer blocks) are followed by
+ * a linear layer, and  LN(x) W^T + b  =  rstd * ((gamma .* x) W^T - mean (gamma W^T)) + (b + beta W^T):  the qkv and
+ * MLP-up GEMMs run on the residual rows scaled by gamma only (rounded to bf16) and apply each row's rstd and mean in
+ * their epilogue, with two constants per output computed at create time, so no normalisation kernel runs inside a block.  The rows' statistics (mean
+ * and squared deviations per 128 columns, merged in index order: independent of sm_budget and of the tile shape) and
+ * their scaled bf16 copy are written by the residual GEMM that produced the rows, in the same pass that adds into the fp32
+ * stream.  on = 0 restores one normalisation kernel per norm1 / norm2 (the result differs in rounding only: the
+ * normalised values are then rounded to bf16 before the GEMM instead of the scaled ones).  While split K is in effect for a
+ * micro-batch its blocks run unfolded.  Both modes stay within the same parity tolerance of the definition. */
+eas_status eas_encoder_set_norm_fold(eas_encoder* enc, int32_t on);
+
 /* Launch-overhead path for small micro-batches (Section 3.2: a forward pass at small batch size is dominated by
  * kernel-launch and scheduling overhead).  mode 1: eas_encode_microbatch / _static capture the launches of a
  * micro-batch into a CUDA graph the first time they see it and replay the graph afterwards (one driver call per

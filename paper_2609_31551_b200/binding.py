@@ -17,7 +17,7 @@ EXPORTED_SYMBOLS = [
     "eas_encoder_create", "eas_encoder_weight_arena_bytes", "eas_encoder_workspace_bytes", "eas_encoder_out_rows",
     "eas_encode_microbatch", "eas_encode_microbatch_static", "eas_encoder_status", "eas_encoder_last_launch_count", "eas_encoder_set_attention_impl",
     "eas_encoder_set_graph_mode", "eas_encoder_graph_stats", "eas_encoder_enable_timing", "eas_encoder_timing_read", "eas_last_error", "eas_encoder_destroy", "eas_kernel_gemm", "eas_kernel_gemm_tile", "eas_kernel_norm", "eas_kernel_attention",
-    "eas_encoder_set_split_k", "eas_sm_partition_create", "eas_sm_partition_sm_count", "eas_sm_partition_stream", "eas_sm_partition_destroy",
+    "eas_encoder_set_split_k", "eas_encoder_set_norm_fold", "eas_sm_partition_create", "eas_sm_partition_sm_count", "eas_sm_partition_stream", "eas_sm_partition_destroy",
 ]
 
 
@@ -80,6 +80,8 @@ def load_library():
     lib.eas_encoder_set_attention_impl.argtypes = [C.c_void_p, C.c_int32]
     lib.eas_encoder_set_split_k.restype = C.c_int
     lib.eas_encoder_set_split_k.argtypes = [C.c_void_p, C.c_int32]
+    lib.eas_encoder_set_norm_fold.restype = C.c_int
+    lib.eas_encoder_set_norm_fold.argtypes = [C.c_void_p, C.c_int32]
     lib.eas_encoder_set_graph_mode.restype = C.c_int
     lib.eas_encoder_set_graph_mode.argtypes = [C.c_void_p, C.c_int32]
     lib.eas_encoder_graph_stats.restype = C.c_int
@@ -253,6 +255,10 @@ class Encoder:
     def set_split_k(self, on: bool):
         """eas_encoder_set_split_k: small micro-batches split the K loop of the residual GEMMs (default off)."""
         _check(self.lib.eas_encoder_set_split_k(self.handle, 1 if on else 0))
+
+    def set_norm_fold(self, on: bool):
+        """eas_encoder_set_norm_fold: the blocks' normalisations inside the GEMMs around them (default on)."""
+        _check(self.lib.eas_encoder_set_norm_fold(self.handle, 1 if on else 0))
 
     def set_graph_mode(self, on: bool):
         """eas_encoder_set_graph_mode: replay captured forward passes for repeated micro-batch shapes.  Needs a

@@ -131,6 +131,8 @@ struct Linear {
 struct Layer {
   const bf16 *n1g = nullptr, *n1b = nullptr, *n2g = nullptr, *n2b = nullptr;
   Linear qkv, proj, fc1, fc2;
+  // folded normalisation (GemmParams::fold_stats): the two per-output constants of the qkv and MLP-up layers
+  const float *qkv_c0 = nullptr, *qkv_c1 = nullptr, *fc1_c0 = nullptr, *fc1_c1 = nullptr;
 };
 
 // One captured forward pass: every launch of a micro-batch with exactly these shapes, pointers and SM budget.
@@ -155,6 +157,7 @@ struct eas_encoder {
   std::vector<Layer> layers;
   int attn_impl = 0;
   int split_k = 0;            // small micro-batches split the K loop of the residual GEMMs (eas_encoder_set_split_k)
+  int fold = 0;               // 1: the blocks' normalisations are folded into the GEMMs around them (eas_encoder_set_norm_fold)
   int last_launches = 0;
   uint32_t* last_status = nullptr;
   // optional per-kernel timing: one event before every launch and one after the last
@@ -228,6 +231,9 @@ extern "C" size_t eas_encoder_weight_arena_bytes(const eas_arch_config* c) {
     total += align_up(d * align_up(embed_k_of(c), 64) * 2, 1024) + align_up(align_up(embed_k_of(c), 64) * 2, 1024);
   if (c->pos == EAS_POS_ROPE_2D) total += c->n_layers * (align_up(3 * d * d * 2, 1024) + align_up(3 * d * 2, 1024));
   if (c->mlp == EAS_MLP_SWIGLU) total += c->n_layers * (align_up(2 * I * d * 2, 1024) + align_up(2 * I * 2, 1024));
+  // folded normalisation: two fp32 constants per output of the qkv and MLP-up layers
+  const size_t n1 = c->mlp == EAS_MLP_SWIGLU ? 2 * I : I;
+  total += c->n_layers * (2 * align_up(3 * d * 4, 1024) + 2 * align_up(n1 * 4, 1024));
   return total;
 }
 
@@ -311,7 +317,14 @@ static eas_status finish_linear(Linear& L) {
 typedef void (*GemmKernel)(GemmParams);
 // ctas: 1 = one CTA per 128x256 tile; 2 = CTA pair per 256x256 tile; 3 = CTA pair per 256x512 tile ("wide");
 // deep (pair tiles only): two 64-wide k-blocks per stage and TMA operation
+// out_fp32: 0 bf16, 1 fp32 (reduce-add when a residual is given), 2 the folding residual epilogue (OUT_F32_FOLD)
 static GemmKernel gemm_kernel_for(int act, int out_fp32, int ctas, bool deep = false, bool split = false) {
+  if (out_fp32 == 2) {
+    if (act != ACT_NONE || split) return nullptr;
+    if (ctas == 3) return gemm_kernel<ACT_NONE, OUT_F32_FOLD, 2, 2>;
+    if (ctas == 2) return deep ? gemm_kernel<ACT_NONE, OUT_F32_FOLD, 2, 1, 2> : gemm_kernel<ACT_NONE, OUT_F32_FOLD, 2, 1>;
+    return gemm_kernel<ACT_NONE, OUT_F32_FOLD, 1, 1>;
+  }
   if (split) {             // split K: the fp32 residual GEMMs only
     if (act != ACT_NONE || !out_fp32) return nullptr;
     if (ctas == 3) return gemm_kernel<ACT_NONE, OUT_F32, 2, 2, 1, true>;
@@ -347,7 +360,7 @@ static eas_status set_kernel_attributes() {
   for (int deep = 0; deep < 2; ++deep)
     for (int ctas = 1; ctas <= 3; ++ctas)
       for (int act = 0; act < 3; ++act)
-        for (int f32 = 0; f32 < 2; ++f32) {
+        for (int f32 = 0; f32 < 3; ++f32) {
           GemmKernel ks = gemm_kernel_for(act, f32, ctas, deep != 0, true);
           if (ks != nullptr) CUDA_TRY(cudaFuncSetAttribute(ks, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmemBytes));
           GemmKernel k = gemm_kernel_for(act, f32, ctas, deep != 0);
@@ -381,6 +394,19 @@ static eas_status device_check(int* sm_count, int* device = nullptr) {
   CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
   if (major != 10) return fail(EAS_ERR_ARCH, "device is compute capability %d.%d; this library is built for 10.x", major, minor);
   *sm_count = sms;
+  return EAS_OK;
+}
+
+// the constants of a linear layer that follows a normalisation (gamma, beta; beta == nullptr for RMSNorm)
+static eas_status fold_linear(Arena& arena, const Linear& src, const bf16* gamma, const bf16* beta, const float** c0, const float** c1) {
+  float* k0 = static_cast<float*>(arena.take(static_cast<size_t>(src.N) * 4));
+  float* k1 = static_cast<float*>(arena.take(static_cast<size_t>(src.N) * 4));
+  if (k0 == nullptr || k1 == nullptr) return fail(EAS_ERR_WORKSPACE, "weight arena exhausted");
+  FoldWeightsParams fp{src.w, src.b, gamma, beta, k0, k1, src.N, src.K};
+  fold_weights_kernel<<<std::min((src.N + 7) / 8, 2048), 256>>>(fp);
+  CUDA_TRY(cudaGetLastError());
+  *c0 = k0;
+  *c1 = k1;
   return EAS_OK;
 }
 
@@ -495,6 +521,8 @@ extern "C" eas_status eas_encoder_create(const eas_arch_config* arch, const eas_
     EAS_TRY(wi.get(p + "fc2.b", {d}, &L.fc2.b));
     L.fc2.N = d; L.fc2.K = I;
     EAS_TRY(finish_linear(L.fc2));
+    EAS_TRY(fold_linear(arena, L.qkv, L.n1g, ln ? L.n1b : nullptr, &L.qkv_c0, &L.qkv_c1));
+    EAS_TRY(fold_linear(arena, L.fc1, L.n2g, ln ? L.n2b : nullptr, &L.fc1_c0, &L.fc1_c1));
   }
   if (c.final_norm) {
     EAS_TRY(wi.get("final_norm.g", {d}, &e->fng));
@@ -531,12 +559,18 @@ extern "C" eas_status eas_encoder_set_split_k(eas_encoder* enc, int32_t on) {
   return EAS_OK;
 }
 
+extern "C" eas_status eas_encoder_set_norm_fold(eas_encoder* enc, int32_t on) {
+  if (enc == nullptr) return fail(EAS_ERR_INVALID_ARG, "encoder is null");
+  enc->fold = on != 0;
+  return EAS_OK;
+}
+
 extern "C" int32_t eas_encoder_last_launch_count(const eas_encoder* enc) { return enc ? enc->last_launches : 0; }
 
 // ------------------------------------------------------------------------------------ workspace plan
 namespace {
 struct Plan {
-  size_t status, x, n, qkv, o, a, row_map, pos_idx, head_src, rope, mel_pad, h1_pad, conv1_map, part, total;
+  size_t status, x, n, qkv, o, a, row_map, pos_idx, head_src, rope, mel_pad, h1_pad, conv1_map, part, stats, total;
   int splits_proj, splits_fc2;     // split-K factors of the two residual GEMMs of a block (1: off)
   int64_t part_rows;               // rows of one split's region of the partial-sum scratch
   int64_t T, embed_rows, padded_rows, out_rows;
@@ -583,6 +617,7 @@ static Plan make_plan(const eas_encoder* e, int64_t T, int n_items) {
   p.splits_fc2 = e->split_k ? pick_splits(T, c.d_model, c.d_mlp, e->sm_count) : 1;
   p.part_rows = (T + 2 * kBM - 1) / (2 * kBM) * (2 * kBM);
   p.part = take(static_cast<size_t>(std::max(p.splits_proj, p.splits_fc2) - 1) * p.part_rows * d * 4);
+  p.stats = take(static_cast<size_t>(T) * (d / kFoldGroup) * 8);    // (mean, M2) per row and group of 128 columns
   p.total = off;
   return p;
 }
@@ -669,6 +704,16 @@ struct GemmCall {
   int64_t part_rows = 0;
   long long rope_stride = 0;   // rows of the [pair][row] table
   int rope_pairs = 0, rope_ncols = 0, head_dim = 0;
+  // folded normalisation (GemmParams::fold_stats).  Consumer: fold_stats with fold_c0 / fold_c1 of the folded weights in
+  // `lin`.  Producer (an in-place fp32 residual GEMM): fold_stats_out, fold_xb and fold_gamma.
+  const float2* fold_stats = nullptr;
+  const float *fold_c0 = nullptr, *fold_c1 = nullptr;
+  int fold_rms = 0;
+  float fold_eps = 0.f;
+  int64_t fold_rows = 0;
+  float2* fold_stats_out = nullptr;
+  bf16* fold_xb = nullptr;
+  const bf16* fold_gamma = nullptr;
 };
 }  // namespace
 
@@ -713,6 +758,12 @@ static eas_status launch_gemm(const GemmCall& g, int budget, cudaStream_t stream
     wide = EAS_GEMM_FORCE_TILE == 3 && tma_out && g.act != ACT_SWIGLU && L.N % 512 == 0 && gemm_kernel_for(g.act, g.out_fp32, 3) != nullptr;
 #endif
   }
+  const bool fold_out = g.fold_stats_out != nullptr;
+  if (fold_out && (!tma_out || !g.out_fp32 || g.resid != g.out || g.splits != 1 || g.act != ACT_NONE || g.fold_xb == nullptr || g.fold_gamma == nullptr || L.N % kFoldGroup != 0))
+    return fail(EAS_ERR_UNSUPPORTED, "the folding epilogue needs an in-place fp32 residual GEMM with N %% %d == 0", kFoldGroup);
+  if (g.fold_stats != nullptr && (!tma_out || g.fold_c0 == nullptr || g.a_run % kFoldGroup != 0 || g.taps != 1))
+    return fail(EAS_ERR_UNSUPPORTED, "a folded normalisation needs a plain GEMM with row-aligned output and K %% %d == 0", kFoldGroup);
+  const int out_mode = fold_out ? 2 : (g.out_fp32 ? 1 : 0);
   const int tile_n = wide ? 2 * kBN : kBN;
   // pair tiles of plain GEMMs run the deep kernel (two k-blocks per stage and TMA operation: 8 % faster at K = 1024);
   // single-CTA and wide tiles would be left with two 96 KB stages and measured no better, and convolutions walk their
@@ -746,6 +797,9 @@ static eas_status launch_gemm(const GemmCall& g, int budget, cudaStream_t stream
   p.row_map = g.row_map; p.pos_idx = g.pos_idx; p.pos = g.pos;
   p.rope_cs = g.rope_cs; p.rope_stride = g.rope_stride; p.rope_pairs = g.rope_pairs; p.rope_ncols = g.rope_ncols; p.head_dim = g.head_dim > 0 ? g.head_dim : 64;
   p.status = status;
+  p.fold_stats = g.fold_stats; p.fold_c0 = g.fold_c0; p.fold_c1 = g.fold_c1; p.fold_rows = g.fold_rows;
+  p.fold_parts = static_cast<int>(g.a_run / kFoldGroup); p.fold_rms = g.fold_rms; p.fold_eps = g.fold_eps;
+  p.fold_stats_out = g.fold_stats_out; p.fold_xb = g.fold_xb; p.fold_gamma = g.fold_gamma;
   // TMA-store epilogue whenever output rows are the A rows and any residual is accumulated in place
   p.use_tma_out = tma_out ? 1 : 0;
   if (p.use_tma_out) {
@@ -753,7 +807,7 @@ static eas_status launch_gemm(const GemmCall& g, int budget, cudaStream_t stream
     EAS_TRY(make_out_tmap(&p.tma_out, g.out, g.out_fp32 != 0, out_cols, g.ldo, g.M));
   }
   const int tiles = p.m_blocks * p.n_blocks * p.splits;
-  GemmKernel kern = gemm_kernel_for(g.act, g.out_fp32, wide ? 3 : ctas, deep, p.splits > 1);
+  GemmKernel kern = gemm_kernel_for(g.act, out_mode, wide ? 3 : ctas, deep, p.splits > 1);
   if (kern == nullptr) return fail(EAS_ERR_UNSUPPORTED, "no GEMM epilogue for act=%d out_fp32=%d", g.act, g.out_fp32);
   return launch_kernel(kern, std::min(budget / ctas, tiles) * ctas, kGemmThreads, kGemmSmemBytes, stream, p, ctas);
 }
@@ -779,6 +833,28 @@ static eas_status launch_norm_nv(const NormParams& p, int budget, cudaStream_t s
   }
 #undef EAS_NORM_CASE
   CUDA_TRY(cudaGetLastError());
+  return EAS_OK;
+}
+
+static eas_status launch_fold_stats(const FoldStatsParams& p, int budget, cudaStream_t stream) {
+  if (p.rows <= 0) return EAS_OK;
+#define EAS_FOLD_CASE(NV_)                                                                                         \
+  case NV_: {                                                                                                      \
+    static OncePerDevice once;                                                                                     \
+    if (once.first()) {                                                                                            \
+      CUDA_TRY(cudaFuncSetAttribute(fold_stats_kernel<NV_>, cudaFuncAttributeMaxDynamicSharedMemorySize, kOnePerSmSmem)); \
+      once.settled();                                                                                              \
+    }                                                                                                              \
+    EAS_TRY(launch_kernel(fold_stats_kernel<NV_>, std::min(budget, (p.rows + 15) / 16), 512, kOnePerSmSmem, stream, p)); \
+    break;                                                                                                         \
+  }
+  switch (p.d / 128) {
+    EAS_FOLD_CASE(1) EAS_FOLD_CASE(2) EAS_FOLD_CASE(3) EAS_FOLD_CASE(4) EAS_FOLD_CASE(5) EAS_FOLD_CASE(6)
+    EAS_FOLD_CASE(7) EAS_FOLD_CASE(8) EAS_FOLD_CASE(9) EAS_FOLD_CASE(10) EAS_FOLD_CASE(11) EAS_FOLD_CASE(12)
+    EAS_FOLD_CASE(13) EAS_FOLD_CASE(14) EAS_FOLD_CASE(15) EAS_FOLD_CASE(16)
+    default: return fail(EAS_ERR_UNSUPPORTED, "row width %d", p.d);
+  }
+#undef EAS_FOLD_CASE
   return EAS_OK;
 }
 
@@ -987,6 +1063,10 @@ static eas_status encode_impl(eas_encoder* e, const eas_packed_inputs* in, void*
   bf16* h1_pad = reinterpret_cast<bf16*>(ws + pl.h1_pad);
   int* conv1_map = reinterpret_cast<int*>(ws + pl.conv1_map);
   float* part = reinterpret_cast<float*>(ws + pl.part);
+  float2* stats = reinterpret_cast<float2*>(ws + pl.stats);
+  // Folded normalisation: the blocks' norm1 / norm2 run inside the GEMMs around them (GemmParams::fold_stats) unless the
+  // residual GEMMs split K, whose partial sums a normalisation kernel has to add.
+  const bool fold = e->fold != 0 && c.n_layers > 0 && pl.splits_proj == 1 && pl.splits_fc2 == 1;
   int pending_parts = 0;      // split-K partial sums of the last residual GEMM, to be added by the next normalisation
   int launches = 0;
   e->last_status = status;
@@ -1074,9 +1154,19 @@ static eas_status encode_impl(eas_encoder* e, const eas_packed_inputs* in, void*
   // Consecutive kernels walk the token rows in alternating directions (`dir`): each starts with the rows its producer
   // wrote last, which are the ones still in L2.  Every row, tile and attention unit is independent of the order.
   int dir = 0;
+  if (fold) {
+    // the first block's rows come from the embedding: their bf16 copy and group statistics from a kernel of its own
+    FoldStatsParams fp{x, nbuf, stats, e->layers[0].n1g, static_cast<int>(T), d};
+    EAS_TRY(mark(e, EAS_KC_NORM, stream));
+    EAS_TRY(launch_fold_stats(fp, budget, stream)); ++launches;
+  }
+  auto fold_in = [&](GemmCall& g, const float* c0, const float* c1) {    // a GEMM on rows scaled by gamma only
+    g.fold_stats = stats; g.fold_c0 = c0; g.fold_c1 = ln_kind == NORM_LN ? c1 : nullptr;
+    g.fold_rms = ln_kind == NORM_RMS ? 1 : 0; g.fold_eps = c.norm_eps; g.fold_rows = T;
+  };
   for (int li = 0; li < c.n_layers; ++li) {
     const Layer& L = e->layers[li];
-    {
+    if (!fold) {
       NormParams np{x, nbuf, L.n1g, L.n1b, nullptr, static_cast<int>(T), d, c.norm_eps};
       np.part = part; np.part_stride = pl.part_rows * d; np.n_part = pending_parts; np.x_rw = x; pending_parts = 0;
       np.reverse = dir; dir ^= 1;
@@ -1086,6 +1176,7 @@ static eas_status encode_impl(eas_encoder* e, const eas_packed_inputs* in, void*
     {
       GemmCall g;
       g.A = nbuf; g.a_run = d; g.a_row_elems = d; g.a_rows = T; g.M = static_cast<int>(T); g.lin = &L.qkv;
+      if (fold) fold_in(g, L.qkv_c0, L.qkv_c1);
       g.out = qkv; g.ldo = 3LL * d;
       if (c.pos == EAS_POS_ROPE_2D) { g.rope_cs = rope; g.rope_stride = T; g.rope_pairs = e->hd / 2; g.rope_ncols = 2 * d; g.head_dim = e->hd; }
       g.reverse = dir; dir ^= 1;
@@ -1100,11 +1191,12 @@ static eas_status encode_impl(eas_encoder* e, const eas_packed_inputs* in, void*
       g.A = obuf; g.a_run = d; g.a_row_elems = d; g.a_rows = T; g.M = static_cast<int>(T); g.lin = &L.proj;
       g.out_fp32 = 1; g.out = x; g.ldo = d; g.resid = x;
       g.splits = pl.splits_proj; g.part = part; g.part_rows = pl.part_rows; pending_parts = g.splits - 1;   // norm2 follows
+      if (fold) { g.fold_stats_out = stats; g.fold_xb = nbuf; g.fold_gamma = L.n2g; g.fold_rows = T; }
       g.reverse = dir; dir ^= 1;
       EAS_TRY(mark(e, EAS_KC_GEMM_PROJ, stream));
       EAS_TRY(launch_gemm(g, budget, stream, status)); ++launches;
     }
-    {
+    if (!fold) {
       NormParams np{x, nbuf, L.n2g, L.n2b, nullptr, static_cast<int>(T), d, c.norm_eps};
       np.part = part; np.part_stride = pl.part_rows * d; np.n_part = pending_parts; np.x_rw = x; pending_parts = 0;
       np.reverse = dir; dir ^= 1;
@@ -1115,6 +1207,7 @@ static eas_status encode_impl(eas_encoder* e, const eas_packed_inputs* in, void*
       GemmCall g;
       g.A = nbuf; g.a_run = d; g.a_row_elems = d; g.a_rows = T; g.M = static_cast<int>(T); g.lin = &L.fc1;
       g.act = c.mlp == EAS_MLP_SWIGLU ? ACT_SWIGLU : ACT_GELU;
+      if (fold) fold_in(g, L.fc1_c0, L.fc1_c1);
       g.out = abuf; g.ldo = c.d_mlp;
       g.reverse = dir; dir ^= 1;
       EAS_TRY(mark(e, EAS_KC_GEMM_FC1, stream));
@@ -1126,6 +1219,7 @@ static eas_status encode_impl(eas_encoder* e, const eas_packed_inputs* in, void*
       g.out_fp32 = 1; g.out = x; g.ldo = d; g.resid = x;
       if (li + 1 < c.n_layers) {      // the next block's first normalisation adds the partial sums
         g.splits = pl.splits_fc2; g.part = part; g.part_rows = pl.part_rows; pending_parts = g.splits - 1;
+        if (fold) { g.fold_stats_out = stats; g.fold_xb = nbuf; g.fold_gamma = e->layers[li + 1].n1g; g.fold_rows = T; }
       }
       g.reverse = dir; dir ^= 1;
       EAS_TRY(mark(e, EAS_KC_GEMM_FC2, stream));

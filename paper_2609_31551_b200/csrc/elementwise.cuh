@@ -134,6 +134,79 @@ __global__ void __launch_bounds__(512, 1) norm_kernel(const NormParams p) {
   }
 }
 
+// ------------------------------------------------------------------------------- folded normalisation: first producer
+// What the residual GEMMs' folding epilogue writes for the rows it updates (GemmParams::fold_stats_out, fold_xb), for
+// rows that come from somewhere else (the embedding): each row scaled by gamma and rounded to bf16 and, per group of 128
+// columns, the mean and the sum of squared deviations from it (of the unscaled values).  One warp per row; lane l holds columns 128 i + 4 l ... + 3 of group i.
+struct FoldStatsParams {
+  const float* x;        // [rows, d]
+  bf16* xb;              // [rows, d]
+  float2* stats;         // [d / 128][rows]
+  const bf16* gamma;     // [d]
+  int rows, d;
+};
+template <int NV>
+__global__ void __launch_bounds__(512, 1) fold_stats_kernel(const FoldStatsParams p) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int warps_per_cta = blockDim.x >> 5;
+  float4 g[NV];
+#pragma unroll
+  for (int i = 0; i < NV; ++i) {
+    const uint2 gv = __ldg(reinterpret_cast<const uint2*>(p.gamma + i * 128 + lane * 4));
+    g[i] = make_float4(bf16_lo(gv.x), bf16_hi(gv.x), bf16_lo(gv.y), bf16_hi(gv.y));
+  }
+  pdl_launch_dependents();
+  pdl_wait();
+  for (int row = blockIdx.x * warps_per_cta + warp; row < p.rows; row += gridDim.x * warps_per_cta) {
+    const float4* xr = reinterpret_cast<const float4*>(p.x + static_cast<long long>(row) * p.d);
+    float4 v[NV];
+#pragma unroll
+    for (int i = 0; i < NV; ++i) v[i] = xr[i * 32 + lane];
+#pragma unroll
+    for (int i = 0; i < NV; ++i) {
+      float s = (v[i].x + v[i].y) + (v[i].z + v[i].w);
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+      const float mean = s * (1.0f / 128.0f);
+      const float a = v[i].x - mean, b = v[i].y - mean, c = v[i].z - mean, e = v[i].w - mean;
+      float q = (a * a + b * b) + (c * c + e * e);
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) q += __shfl_xor_sync(0xffffffffu, q, o);
+      if (lane == 0) p.stats[static_cast<long long>(i) * p.rows + row] = make_float2(mean, q);
+      reinterpret_cast<uint2*>(p.xb + static_cast<long long>(row) * p.d)[i * 32 + lane] =
+          make_uint2(pack_bf16x2(v[i].x * g[i].x, v[i].y * g[i].y), pack_bf16x2(v[i].z * g[i].z, v[i].w * g[i].w));
+    }
+  }
+}
+
+// Create time: the two per-output constants of GemmParams::fold_stats for a linear layer that follows a normalisation.
+// One warp per weight row.
+struct FoldWeightsParams {
+  const bf16* w;         // [n, k]
+  const bf16* bias;      // [n]
+  const bf16* gamma;     // [k]
+  const bf16* beta;      // [k] or nullptr (RMSNorm)
+  float* c0;             // [n]     bias[n] + sum_k beta_k * w[n, k]
+  float* c1;             // [n]     sum_k gamma_k * w[n, k]
+  int n, k;
+};
+__global__ void __launch_bounds__(256) fold_weights_kernel(const FoldWeightsParams p) {
+  const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+  const int n_warps = (gridDim.x * blockDim.x) >> 5;
+  for (int row = warp; row < p.n; row += n_warps) {
+    const bf16* wr = p.w + static_cast<long long>(row) * p.k;
+    float s1 = 0.f, s0 = 0.f;
+    for (int j = lane; j < p.k; j += 32) {
+      const float w = __bfloat162float(wr[j]);
+      s1 = fmaf(w, __bfloat162float(p.gamma[j]), s1);
+      if (p.beta != nullptr) s0 = fmaf(w, __bfloat162float(p.beta[j]), s0);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) { s1 += __shfl_xor_sync(0xffffffffu, s1, o); s0 += __shfl_xor_sync(0xffffffffu, s0, o); }
+    if (lane == 0) { p.c1[row] = s1; p.c0[row] = s0 + __bfloat162float(p.bias[row]); }
+  }
+}
+
 // ------------------------------------------------------------------------------- per-call tables
 struct PrepParams {
   ItemTable items;

@@ -51,7 +51,11 @@ constexpr int kTmemCols = 512;
 constexpr int kPanelM = 8;                        // m-blocks per rasterisation panel (L2 reuse of W tiles)
 
 enum { ACT_NONE = 0, ACT_GELU = 1, ACT_SWIGLU = 2 };
-enum { OUT_BF16 = 0, OUT_F32 = 1 };
+// OUT_F32_FOLD: the fp32 residual update x = x + A W^T + b done in the epilogue's registers (instead of a reduce-add
+// in L2), so that the same pass also writes the bf16 copy of the new rows and their statistics: what the next GEMM's
+// folded normalisation reads (see GemmParams::fold_stats).
+enum { OUT_BF16 = 0, OUT_F32 = 1, OUT_F32_FOLD = 2 };
+constexpr int kFoldGroup = 128;                   // columns per statistics group
 
 struct alignas(64) GemmParams {
   CUtensorMap tma_a;      // 3-D: {K-run, phase, rows}; box {64, 1, 128}.  Deep kernels: {64, rows, K/64}; box {64, 128, 2}
@@ -86,6 +90,23 @@ struct alignas(64) GemmParams {
   int kb_per_split;
   int part_rows;          // rows of one split's region of the scratch matrix (a multiple of the tile height)
   CUtensorMap tma_part;   // [(splits - 1) * part_rows, N] fp32, 32-row boxes of 32 columns
+  // Folded normalisation.  LayerNorm / RMSNorm followed by a linear layer is  rstd * ((gamma .* x) - mean gamma) W^T + const:
+  // the GEMM can run on the rows scaled by gamma only (rounded to bf16: the same single rounding of the operand as
+  // with a normalisation kernel) and apply the row's rstd and mean in its epilogue,
+  //     out[i, n] = rstd_i * (acc[i, n] - mean_i * c1[n]) + c0[n],   c1[n] = sum_k gamma_k W[n, k],  c0[n] = b[n] + sum_k beta_k W[n, k],
+  // so no normalisation kernel runs between the residual GEMM and this one.  The statistics arrive as one (mean, M2)
+  // pair per row and group of kFoldGroup columns (M2 = sum of squared deviations from the group's mean), written by
+  // the producer of the rows, and are merged in index order: budget- and tile-shape-independent.
+  const float2* fold_stats;   // consumer: [fold_parts][fold_rows]; nullptr = no folding
+  const float* fold_c0;       // consumer: [N] fp32, replaces bias
+  const float* fold_c1;       // consumer: [N] fp32 (LayerNorm; nullptr for RMSNorm, which subtracts no mean)
+  long long fold_rows;        // rows of one group's slab of the statistics (both sides)
+  int fold_parts;             // groups per row: K / kFoldGroup
+  int fold_rms;               // 1: rstd from the mean square; 0: from the variance
+  float fold_eps;
+  float2* fold_stats_out;     // producer (OUT_F32_FOLD): [N / kFoldGroup][fold_rows]
+  bf16* fold_xb;              // producer: bf16(gamma .* updated rows), [*, ldo]
+  const bf16* fold_gamma;     // producer: [N], the gamma of the normalisation the rows go through next
   uint32_t* status;       // device status word
 };
 
@@ -318,10 +339,41 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_kernel(const __grid_cons
 #pragma unroll
           for (int h = 0; h < NW; ++h) {
             const int col = nb * kTileN + h * 256 + ew * 32 + lane;
-            sbias[h * 256 + ew * 32 + lane] = (col < p.N && split == 0) ? __bfloat162float(p.bias[col]) : 0.f;
+            sbias[h * 256 + ew * 32 + lane] = (col < p.N && split == 0) ? (p.fold_stats != nullptr ? p.fold_c0[col] : __bfloat162float(p.bias[col])) : 0.f;
           }
           __syncwarp();
           if (lane == 0) mbar_arrive(&bias_bar[acc]);
+        }
+        // folded normalisation: this thread's row factor and offset, from the row's group statistics (loaded while the
+        // tile's main loop is still running)
+        float fold_a = 1.f, fold_b = 0.f;
+        if (p.fold_stats != nullptr) {
+          const long long r = min(mb * kBM + quarter * 32 + lane, p.M - 1);
+          float mu = 0.f, m2 = 0.f;
+          for (int g = 0; g < p.fold_parts; ++g) {       // groups of equal size, merged in index order
+            const float2 st = __ldg(p.fold_stats + g * p.fold_rows + r);
+            const float delta = st.x - mu;
+            const float inv = 1.0f / static_cast<float>(g + 1);
+            mu += delta * inv;
+            m2 += st.y + delta * delta * (static_cast<float>(kFoldGroup * g) * inv);
+          }
+          const float inv_k = 1.0f / static_cast<float>(kFoldGroup * p.fold_parts);
+          if (p.fold_rms) {
+            fold_a = 1.0f / sqrtf((m2 * inv_k + mu * mu) + p.fold_eps);
+          } else {
+            fold_a = 1.0f / sqrtf(m2 * inv_k + p.fold_eps);
+            fold_b = -fold_a * mu;
+          }
+        }
+        if (OUT == OUT_F32_FOLD) {
+          // the rows this tile updates, towards L2 while the main loop runs (the epilogue reads them with plain loads)
+          const int r = mb * kBM + quarter * 32 + lane;
+          if (r < p.M) {
+            const char* base = reinterpret_cast<const char*>(p.resid + static_cast<long long>(r) * p.ldo + nb * kTileN + half * (128 * NW));
+#pragma unroll
+            for (int i = 0; i < 4 * NW; ++i)
+              if (nb * kTileN + half * (128 * NW) + i * 32 < p.N) asm volatile("prefetch.global.L2 [%0];" ::"l"(base + i * 128));
+          }
         }
         GEMM_STAMP(0);
         if (!mbar_wait(&acc_full[acc], acc_ph, abort_flag)) { ok = false; break; }
@@ -340,10 +392,26 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_kernel(const __grid_cons
         auto finish_chunk = [&](float (&v)[32], int c) {   // bias, rotary, activation on 32 accumulator columns
           const int col0 = nb * kTileN + half * (128 * NW) + c * 32;
           const float4* b4 = reinterpret_cast<const float4*>(sbias + half * (128 * NW) + c * 32);
+          if (p.fold_stats != nullptr) {
+            // out = rstd * acc + (c0 - rstd * mean * c1): the staged "bias" is c0
+            const bool centred = p.fold_c1 != nullptr && col0 < p.N;
+            const float4* c4 = reinterpret_cast<const float4*>(p.fold_c1 + (centred ? col0 : 0));
 #pragma unroll
-          for (int q = 0; q < 8; ++q) {
-            const float4 b = b4[q];
-            v[4 * q] += b.x; v[4 * q + 1] += b.y; v[4 * q + 2] += b.z; v[4 * q + 3] += b.w;
+            for (int q = 0; q < 8; ++q) {
+              float4 b = b4[q];
+              if (centred) {
+                const float4 c1 = __ldg(c4 + q);
+                b.x = fmaf(fold_b, c1.x, b.x); b.y = fmaf(fold_b, c1.y, b.y); b.z = fmaf(fold_b, c1.z, b.z); b.w = fmaf(fold_b, c1.w, b.w);
+              }
+              v[4 * q] = fmaf(fold_a, v[4 * q], b.x); v[4 * q + 1] = fmaf(fold_a, v[4 * q + 1], b.y);
+              v[4 * q + 2] = fmaf(fold_a, v[4 * q + 2], b.z); v[4 * q + 3] = fmaf(fold_a, v[4 * q + 3], b.w);
+            }
+          } else {
+#pragma unroll
+            for (int q = 0; q < 8; ++q) {
+              const float4 b = b4[q];
+              v[4 * q] += b.x; v[4 * q + 1] += b.y; v[4 * q + 2] += b.z; v[4 * q + 3] += b.w;
+            }
           }
           if (p.rope_cs != nullptr && col0 < p.rope_ncols && arow < p.M) {
             int pi = (col0 % p.head_dim) >> 1;
@@ -387,7 +455,86 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_kernel(const __grid_cons
           }
         };
 
-        if (OUT == OUT_F32) {
+        if (OUT == OUT_F32_FOLD) {
+          // x = x + A W^T + b in registers, one 32-column chunk per round: the old values by plain loads (one chunk
+          // ahead, prefetched towards L2 before the main loop ended), the new ones through the staging buffer and a
+          // TMA store; the bf16 copy (scaled by the next normalisation's gamma) straight from registers; the chunk's mean and squared deviations merged into its
+          // 128-column group, written when the group is complete.
+          static_assert(OUT != OUT_F32_FOLD || ACT == ACT_NONE, "the folding residual epilogue has no activation");
+          constexpr int kChunks = 4 * NW;
+          const bool row_ok = arow < p.M;
+          const int tcol0 = nb * kTileN + half * (128 * NW);
+          const long long roff = static_cast<long long>(row_ok ? arow : 0) * p.ldo + tcol0;
+          const float4* xin = reinterpret_cast<const float4*>(p.resid + roff);
+          uint4* xb = reinterpret_cast<uint4*>(p.fold_xb + roff);
+          const float4* b4 = reinterpret_cast<const float4*>(sbias + half * (128 * NW));
+          uint32_t r[32];
+          float4 xo[8];
+          __syncwarp();
+          tmem_ld_32x32(taddr, r);
+#pragma unroll
+          for (int q = 0; q < 8; ++q) xo[q] = (row_ok && tcol0 < p.N) ? __ldcg(xin + q) : make_float4(0.f, 0.f, 0.f, 0.f);
+          float gm = 0.f, gm2 = 0.f;
+#pragma unroll 1
+          for (int c = 0; c < kChunks; ++c) {
+            tmem_ld_wait();
+            float v[32];
+#pragma unroll
+            for (int q = 0; q < 8; ++q) {
+              const float4 b = b4[c * 8 + q];
+              v[4 * q] = (__uint_as_float(r[4 * q]) + b.x) + xo[q].x;
+              v[4 * q + 1] = (__uint_as_float(r[4 * q + 1]) + b.y) + xo[q].y;
+              v[4 * q + 2] = (__uint_as_float(r[4 * q + 2]) + b.z) + xo[q].z;
+              v[4 * q + 3] = (__uint_as_float(r[4 * q + 3]) + b.w) + xo[q].w;
+            }
+            const int col0 = tcol0 + c * 32;
+            if (c + 1 < kChunks) {
+              __syncwarp();
+              tmem_ld_32x32(taddr + (c + 1) * 32, r);
+              const bool more = row_ok && col0 + 32 < p.N;
+#pragma unroll
+              for (int q = 0; q < 8; ++q) xo[q] = more ? __ldcg(xin + (c + 1) * 8 + q) : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+            // the chunk's statistics (two passes over registers), merged into the group's (counts 32 k and 32)
+            float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+#pragma unroll
+            for (int i = 0; i < 32; i += 4) { s0 += v[i]; s1 += v[i + 1]; s2 += v[i + 2]; s3 += v[i + 3]; }
+            const float cm = ((s0 + s1) + (s2 + s3)) * (1.0f / 32.0f);
+            float q0 = 0.f, q1 = 0.f;
+#pragma unroll
+            for (int i = 0; i < 32; i += 2) {
+              const float t0 = v[i] - cm, t1 = v[i + 1] - cm;
+              q0 = fmaf(t0, t0, q0); q1 = fmaf(t1, t1, q1);
+            }
+            const int k = c & 3;
+            if (k == 0) {
+              gm = cm; gm2 = q0 + q1;
+            } else {
+              const float delta = cm - gm;
+              const float inv = 1.0f / static_cast<float>(k + 1);
+              gm += delta * inv;
+              gm2 += (q0 + q1) + delta * delta * (static_cast<float>(32 * k) * inv);
+            }
+            if (k == 3 && row_ok && col0 < p.N)
+              p.fold_stats_out[static_cast<long long>(col0 / kFoldGroup) * p.fold_rows + arow] = make_float2(gm, gm2);
+            staging_free();
+#pragma unroll
+            for (int q = 0; q < 8; ++q)
+              *reinterpret_cast<float4*>(srow + ((q ^ sw) << 4)) = make_float4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
+            if (col0 < p.N) store_subtile(col0);
+            if (row_ok && col0 < p.N) {
+              const uint4* g4 = reinterpret_cast<const uint4*>(p.fold_gamma + col0);
+#pragma unroll
+              for (int q = 0; q < 4; ++q) {
+                const uint4 g = __ldg(g4 + q);
+                xb[c * 4 + q] = make_uint4(pack_bf16x2(v[8 * q] * bf16_lo(g.x), v[8 * q + 1] * bf16_hi(g.x)),
+                                           pack_bf16x2(v[8 * q + 2] * bf16_lo(g.y), v[8 * q + 3] * bf16_hi(g.y)),
+                                           pack_bf16x2(v[8 * q + 4] * bf16_lo(g.z), v[8 * q + 5] * bf16_hi(g.z)),
+                                           pack_bf16x2(v[8 * q + 6] * bf16_lo(g.w), v[8 * q + 7] * bf16_hi(g.w)));
+              }
+            }
+          }
+        } else if (OUT == OUT_F32) {
           // fp32 output: 32 columns = one 128-byte staging row, so every 32-column chunk is a sub-tile (and a TMA
           // operation) of its own.  One chunk per round, the next chunk's TMEM load in flight meanwhile, so that the
           // wait for the previous operation to release the staging buffer falls behind a load and the chunk's math.
@@ -564,7 +711,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_kernel(const __grid_cons
             }
           }
         }
-        if (OUT == OUT_F32) {
+        if (OUT != OUT_BF16) {
           float* o = reinterpret_cast<float*>(p.out) + orow * p.ldo + col0;
           if (p.resid != nullptr) {
             const float4* r4 = reinterpret_cast<const float4*>(p.resid + orow * p.ldo + col0);

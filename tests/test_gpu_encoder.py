@@ -41,6 +41,35 @@ def test_encoder_parity_small(case, profile):
     print(f"{case}/{profile}: row-rel {rel:.3e} max-abs {mabs:.3e}")
 
 
+@pytest.mark.parametrize("case", ["c0_full", "c1_2layers", "c2_2layers", "c3_2layers", "c4_2layers"])
+def test_folded_normalisation_parity_and_determinism(case):
+    """eas_encoder_set_norm_fold: the blocks' normalisations applied inside the GEMMs around them (no normalisation
+    kernel inside a block).  Same tolerance against the oracle as the default path, the same bytes for every SM
+    budget and for an item alone or packed, fewer launches, and switching it off restores the default path's bytes."""
+    name, over, shapes = CASES[case]
+    cfg = S.get_config(name, **over)
+    w, enc = _make(cfg, "sharp")
+    items = S.make_items(cfg, shapes, seed=2050 + len(shapes))
+    ref, _, _ = O.encode_microbatch(cfg, w, items)
+    plain, plain_dev = G.run_gpu(enc, cfg, items)
+    n_plain = enc.last_launch_count()
+    enc.set_norm_fold(True)
+    got, dev = G.run_gpu(enc, cfg, items)
+    rel, mabs = G.assert_parity(got, ref, case + " folded")
+    G.record_margin(f"{case}, folded normalisation", "sharp", 2050 + len(shapes), rel, mabs)
+    assert enc.last_launch_count() == n_plain - 2 * cfg["n_layers"] + 1
+    assert np.abs(got - plain).max() <= G.ABS_TOL          # two roundings of the same values
+    for budget in (3, 37, 111):
+        _, again = G.run_gpu(enc, cfg, items, sm_budget=budget)
+        assert torch.equal(dev, again), budget
+    sl0 = S.out_tokens_per_item(cfg, G.item_shape(cfg, items[0]))
+    _, alone = G.run_gpu(enc, cfg, [items[0]])
+    assert torch.equal(alone, dev[:sl0])
+    enc.set_norm_fold(False)
+    _, back = G.run_gpu(enc, cfg, items)
+    assert torch.equal(back, plain_dev)
+
+
 def test_c0_bit_stability_and_packing_invariance():
     cfg = S.get_config("c0")
     w, enc = _make(cfg)

@@ -42,6 +42,20 @@ def test_c1_bench_configuration_sampled_items():
     assert torch.equal(alone, out_dev[sl[17]])
 
 
+@pytest.mark.parametrize("name,shapes,seed", [("c1", [(1, 336, 336)] * 2, 2121),
+                                               ("c2", [(1, 224, 224), (1, 448, 336)], 2221)])
+def test_full_depth_with_folded_normalisation(name, shapes, seed):
+    """Full depth with eas_encoder_set_norm_fold on: LayerNorm (c1) and RMSNorm with rotary positions (c2)."""
+    cfg = S.get_config(name)
+    w, enc = _make(cfg, "sharp")
+    enc.set_norm_fold(True)
+    items = S.make_items(cfg, shapes, seed=seed)
+    ref, _, _ = O.encode_microbatch(cfg, w, items)
+    got, _ = G.run_gpu(enc, cfg, items)
+    rel, mabs = G.assert_parity(got, ref, f"{name} folded")
+    G.record_margin(f"{name} full depth, folded normalisation", "sharp", seed, rel, mabs)
+
+
 @pytest.mark.parametrize("profile,seed", [("sharp", 2101), ("sharp", 2111), ("plain", 2112)])
 def test_c1_full_depth_two_images(profile, seed):
     cfg = S.get_config("c1")
