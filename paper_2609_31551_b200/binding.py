@@ -257,7 +257,7 @@ class Encoder:
         _check(self.lib.eas_encoder_set_split_k(self.handle, 1 if on else 0))
 
     def set_norm_fold(self, on: bool):
-        """eas_encoder_set_norm_fold: the blocks' normalisations inside the GEMMs around them (default on)."""
+        """eas_encoder_set_norm_fold: the blocks' normalisations inside the GEMMs around them (default off)."""
         _check(self.lib.eas_encoder_set_norm_fold(self.handle, 1 if on else 0))
 
     def set_graph_mode(self, on: bool):
