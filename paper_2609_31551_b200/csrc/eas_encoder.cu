@@ -1282,7 +1282,7 @@ static eas_status encode_cached(eas_encoder* e, const eas_packed_inputs* in, voi
   const int n = in->n_items;
   std::vector<int64_t> key;
   key.reserve(8 + 5 * static_cast<size_t>(n) + 1);
-  key.push_back(n); key.push_back(sm_budget); key.push_back(e->attn_impl * 2 + e->split_k);
+  key.push_back(n); key.push_back(sm_budget); key.push_back(e->attn_impl * 4 + e->split_k * 2 + e->fold);
   key.push_back(static_cast<int64_t>(reinterpret_cast<uintptr_t>(in->data)));
   key.push_back(static_cast<int64_t>(reinterpret_cast<uintptr_t>(workspace)));
   key.push_back(static_cast<int64_t>(workspace_bytes));

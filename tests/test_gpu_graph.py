@@ -61,6 +61,37 @@ def test_graph_replay_is_bit_identical(cfg_name, shapes):
     assert not torch.equal(ref, ref2)
 
 
+def test_graph_mode_follows_the_normalisation_mode():
+    """A captured forward pass belongs to the normalisation mode it was captured in: switching
+    eas_encoder_set_norm_fold between calls must not replay the other mode's launches."""
+    P, cfg, enc, items, data, offsets, cu = _setup("c0", [(1, 224, 224)] * 2, seed=31)
+    shapes = [(1, 224, 224)] * 2
+    cu_dev = torch.from_numpy(cu).cuda()
+    plain = enc.encode_microbatch(data, shapes, offsets, cu, cu_seqlens_dev=cu_dev).clone()
+    enc.set_norm_fold(True)
+    folded = enc.encode_microbatch(data, shapes, offsets, cu, cu_seqlens_dev=cu_dev).clone()
+    n_folded = enc.last_launch_count()
+    enc.set_norm_fold(False)
+    enc.status()
+    assert not torch.equal(plain, folded)                      # two roundings of the same values
+    ws = torch.empty(enc.workspace_bytes(int(cu[-1]), 2) + 1024, dtype=torch.uint8, device="cuda")
+    out = torch.zeros_like(plain)
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    enc.set_graph_mode(True)
+    with torch.cuda.stream(side):
+        for fold, want in ((False, plain), (True, folded), (False, plain), (True, folded)):
+            enc.set_norm_fold(fold)
+            out.zero_()
+            enc.encode_microbatch(data, shapes, offsets, cu, cu_seqlens_dev=cu_dev, out=out, workspace=ws, stream=side)
+            enc.status(side)
+            assert torch.equal(out, want), fold
+            if fold:
+                assert enc.last_launch_count() == n_folded
+    assert enc.graph_stats() == {"hits": 2, "captures": 2, "cached": 2}
+    enc.set_graph_mode(False)
+
+
 def test_graph_cache_keys_on_shape_budget_and_pointers():
     P, cfg, enc, items, data, offsets, cu = _setup("c0", [(1, 224, 224)] * 3, seed=5)
     cu_dev = torch.from_numpy(cu).cuda()
