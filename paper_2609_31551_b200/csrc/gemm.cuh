@@ -131,6 +131,23 @@ __device__ __forceinline__ void tile_coords(int tile, int m_blocks, int n_blocks
   mb = panel * kPanelM + (within - nb * rows_here);
 }
 
+// Folded normalisation: a row's factor and offset (rstd, -rstd * mean) from its group statistics, merged in index
+// order (groups of equal size).  Kept out of line: the GEMM kernels sit at their register limit.
+__device__ __noinline__ float2 fold_row_factors(const float2* stats, long long rows, int parts, int rms, float eps, long long r) {
+  float mu = 0.f, m2 = 0.f;
+  for (int g = 0; g < parts; ++g) {
+    const float2 st = __ldg(stats + g * rows + r);
+    const float delta = st.x - mu;
+    const float inv = 1.0f / static_cast<float>(g + 1);
+    mu += delta * inv;
+    m2 += st.y + delta * delta * (static_cast<float>(kFoldGroup * g) * inv);
+  }
+  const float inv_k = 1.0f / static_cast<float>(kFoldGroup * parts);
+  if (rms) return make_float2(1.0f / sqrtf((m2 * inv_k + mu * mu) + eps), 0.f);
+  const float a = 1.0f / sqrtf(m2 * inv_k + eps);
+  return make_float2(a, -a * mu);
+}
+
 // SPLIT: the launch splits K (GemmParams::splits > 1); the ordinary instantiations keep their code free of it.
 template <int ACT, int OUT, int CTAS, int NW, int KD = 1, bool SPLIT = false>
 __global__ void __launch_bounds__(kGemmThreads, 1) gemm_kernel(const __grid_constant__ GemmParams p) {
@@ -348,22 +365,9 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_kernel(const __grid_cons
         // tile's main loop is still running)
         float fold_a = 1.f, fold_b = 0.f;
         if (p.fold_stats != nullptr) {
-          const long long r = min(mb * kBM + quarter * 32 + lane, p.M - 1);
-          float mu = 0.f, m2 = 0.f;
-          for (int g = 0; g < p.fold_parts; ++g) {       // groups of equal size, merged in index order
-            const float2 st = __ldg(p.fold_stats + g * p.fold_rows + r);
-            const float delta = st.x - mu;
-            const float inv = 1.0f / static_cast<float>(g + 1);
-            mu += delta * inv;
-            m2 += st.y + delta * delta * (static_cast<float>(kFoldGroup * g) * inv);
-          }
-          const float inv_k = 1.0f / static_cast<float>(kFoldGroup * p.fold_parts);
-          if (p.fold_rms) {
-            fold_a = 1.0f / sqrtf((m2 * inv_k + mu * mu) + p.fold_eps);
-          } else {
-            fold_a = 1.0f / sqrtf(m2 * inv_k + p.fold_eps);
-            fold_b = -fold_a * mu;
-          }
+          const float2 f = fold_row_factors(p.fold_stats, p.fold_rows, p.fold_parts, p.fold_rms, p.fold_eps,
+                                            min(mb * kBM + quarter * 32 + lane, p.M - 1));
+          fold_a = f.x; fold_b = f.y;
         }
         if (OUT == OUT_F32_FOLD) {
           // the rows this tile updates, towards L2 while the main loop runs (the epilogue reads them with plain loads)
