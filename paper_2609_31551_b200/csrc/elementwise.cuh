@@ -80,7 +80,7 @@ __global__ void __launch_bounds__(512, 1) norm_kernel(const NormParams p) {
     const float4* xr = reinterpret_cast<const float4*>(p.x + src * p.d);
     float4 v[NV];
 #pragma unroll
-    for (int i = 0; i < NV; ++i) v[i] = xr[i * 32 + lane];
+    for (int i = 0; i < NV; ++i) v[i] = __ldcs(xr + i * 32 + lane);    // streaming: the rows are not read again before they are rewritten
     if (PART) {
       for (int s = 0; s < p.n_part; ++s) {
         const float4* pr = reinterpret_cast<const float4*>(p.part + s * p.part_stride + src * p.d);
